@@ -1,0 +1,125 @@
+"""ctypes access to the CPU oracle (test infrastructure only).
+
+Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
+import this package. The product package never does.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "moesched_oracle.cpp")
+_SO = os.path.join(_HERE, "libmoesched_oracle.so")
+
+MODEL_FIELDS = ("bytes_per_token", "link_gbps", "reconfig_ns", "expert_fixed_ns", "expert_ps_per_token")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no CUDA involved)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _SO, _SRC]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_assignment_max.restype = ctypes.c_int64
+    return _lib
+
+
+def hardware_threads() -> int:
+    return max(1, len(os.sched_getaffinity(0)))
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def mw_decompose(demand, k_max, tier=1, threads=1, want_residual=True):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    perm = np.zeros((B, k_max, N), np.uint8)
+    dur = np.zeros((B, k_max), np.int32)
+    count = np.zeros(B, np.int32)
+    status = np.zeros(B, np.int32)
+    residual = np.zeros_like(d) if want_residual else None
+    rc = lib().oracle_mw_decompose(B, N, _p(d), k_max, _p(perm), _p(dur), _p(count), _p(residual),
+                                   _p(status), tier, threads)
+    if rc != 0:
+        raise ValueError("oracle_mw_decompose rejected its arguments")
+    return dict(perm=perm, dur=dur, count=count, residual=residual, status=status)
+
+
+def bvn_decompose(demand, k_max, tier=1, threads=1, want_aug=True):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    perm = np.zeros((B, k_max, N), np.uint8)
+    coef = np.zeros((B, k_max), np.int32)
+    count = np.zeros(B, np.int32)
+    status = np.zeros(B, np.int32)
+    aug = np.zeros_like(d) if want_aug else None
+    rc = lib().oracle_bvn_decompose(B, N, _p(d), k_max, _p(perm), _p(coef), _p(count), _p(aug),
+                                    _p(status), tier, threads)
+    if rc != 0:
+        raise ValueError("oracle_bvn_decompose rejected its arguments")
+    return dict(perm=perm, coef=coef, count=count, aug=aug, status=status)
+
+
+def schedule_eval(demand, perm, dur, count, model, threads=1):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    perm = np.ascontiguousarray(perm, dtype=np.uint8)
+    dur = np.ascontiguousarray(dur, dtype=np.int32)
+    count = np.ascontiguousarray(count, dtype=np.int32)
+    k_stride = perm.shape[1]
+    m = np.array([int(model[f]) for f in MODEL_FIELDS], np.int64)
+    out = {k: np.zeros(B, np.int64) for k in
+           ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",
+            "unserved_tokens")}
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_schedule_eval(B, N, _p(d), k_stride, _p(perm), _p(dur), _p(count), _p(m),
+                                    _p(out["makespan_overlap_ns"]), _p(out["makespan_serial_ns"]),
+                                    _p(out["compute_idle_ns"]), _p(out["link_idle_tokens"]),
+                                    _p(out["unserved_tokens"]), _p(status), threads)
+    if rc != 0:
+        raise ValueError("oracle_schedule_eval rejected its arguments")
+    out["status"] = status
+    return out
+
+
+def max_weight_perm(W, tier):
+    W = np.ascontiguousarray(W, dtype=np.int64)
+    N = W.shape[0]
+    perm = np.zeros(N, np.int32)
+    rc = lib().oracle_max_weight_perm(N, _p(W), _p(perm), tier)
+    return perm if rc == 0 else None
+
+
+def support_perm(A, tier):
+    A = np.ascontiguousarray(A, dtype=np.int64)
+    N = A.shape[0]
+    perm = np.zeros(N, np.int32)
+    rc = lib().oracle_support_perm(N, _p(A), _p(perm), tier)
+    return perm if rc == 0 else None
+
+
+def assignment_max(W):
+    W = np.ascontiguousarray(W, dtype=np.int64)
+    return int(lib().oracle_assignment_max(W.shape[0], _p(W)))
+
+
+def augment(D):
+    D = np.ascontiguousarray(D, dtype=np.int32)
+    A = np.zeros(D.shape, np.int64)
+    rc = lib().oracle_augment(D.shape[0], _p(D), _p(A))
+    return A if rc == 0 else None
