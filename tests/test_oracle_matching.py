@@ -115,8 +115,9 @@ def test_lexicographic_rule_on_a_worked_case():
 def test_pins_separate_plausible_mistakes():
     """Plausible wrong variants of the rule give a different answer on these inputs,
     so a test above fails if the oracle implements one of them."""
-    W = np.array([[1, 9, 0], [5, 5, 0], [0, 0, 0]])
+    W = np.array([[1, 9, 0], [0, 0, 0], [5, 5, 0]])
     _, arg = brute_max_weight(W)
+    assert arg == [1, 2, 0] and list(oracle.max_weight_perm(W, 1)) == arg
     assert list(oracle.max_weight_perm(W.T.copy(), 1)) != arg      # transposed operand
     assert list(oracle.max_weight_perm(-W, 1)) != arg              # minimising instead of maximising
     # row-by-row argmax is not an optimal matching: rows 0 and 1 both want column 0
