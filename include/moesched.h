@@ -1,0 +1,184 @@
+/*
+ * moesched -- batched circuit scheduling of MoE all-to-all demand matrices on
+ * one NVIDIA B200 (sm_100a).
+ *
+ * For B independent N x N matrices of token counts (demand[b][i][j] = tokens
+ * that rank i sends to rank j) the library computes, entirely on the GPU,
+ *   - the greedy max-weight decomposition           (paper Sec. 3.2),
+ *   - the Birkhoff-von Neumann decomposition        (paper Sec. 3.1),
+ *   - the makespan of such a schedule under the dispatch -> expert compute ->
+ *     combine pipeline with and without overlap     (paper Sec. 4.1, Sec. 3.3).
+ *
+ * Conventions shared by all entry points
+ *   - Plain C ABI. Pointers named d_* are DEVICE pointers, h_* are HOST
+ *     pointers. The caller owns every buffer; the library allocates nothing,
+ *     frees nothing and never synchronises: work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*, NULL = default stream) and the call
+ *     returns at once. Buffers must stay alive until the stream has drained.
+ *   - Matrices are int32, row major, [B][N][N], densely packed. 1 <= N <= 256.
+ *     d_demand should be 16-byte aligned (it then takes the bulk-copy path for
+ *     even N; any 4-byte aligned pointer is still accepted).
+ *   - A matching is a permutation pi stored as N bytes: pi[i] = destination
+ *     rank of source rank i. Schedules are [B][k_max][N] uint8 plus
+ *     [B][k_max] int32 durations (in tokens); only the first count[b]
+ *     matchings of matrix b are written.
+ *   - Tie rule: where several permutations are optimal the lexicographically
+ *     smallest one is returned (row 0 gets the lowest column that any optimal
+ *     matching allows, then row 1, ...). Results are therefore unique and
+ *     independent of the solver.
+ *   - Return value: MOESCHED_OK when the work was enqueued; MOESCHED_EINVAL
+ *     for a null pointer or an out-of-range size (nothing enqueued);
+ *     MOESCHED_ECUDA when a CUDA call failed (moesched_last_cuda_error()).
+ *   - Per-matrix outcome in d_status[b]:
+ *       MOESCHED_ST_OK          complete result
+ *       MOESCHED_ST_TRUNCATED   k_max matchings written, matrix not exhausted
+ *       MOESCHED_ST_BAD_INPUT   matrix b violates the input range; count = 0
+ *       MOESCHED_ST_INTERNAL    an internal iteration limit was hit (a bug)
+ *     No input makes a kernel trap, spin or read out of bounds.
+ */
+#ifndef MOESCHED_H_
+#define MOESCHED_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOESCHED_OK 0
+#define MOESCHED_EINVAL (-1)
+#define MOESCHED_ECUDA (-2)
+
+#define MOESCHED_ST_OK 0
+#define MOESCHED_ST_TRUNCATED 1
+#define MOESCHED_ST_BAD_INPUT (-1)
+#define MOESCHED_ST_INTERNAL (-2)
+
+#define MOESCHED_MAX_N 256
+
+/* Number of int64 work counters per matrix written to d_work (see below). */
+#define MOESCHED_WORK_FIELDS 8
+
+/* Link and compute model of the overlap pipeline (paper Sec. 4.1 "Execution
+ * time"): a matching lasts as long as its largest transfer at link speed; an
+ * expert batch costs a fixed overhead plus a per-token cost (the affine form
+ * of the "knee" of Fig. 1); circuits are reconfigured before every matching.
+ * All integers. Ranges: 1 <= bytes_per_token <= 2^20, 1 <= link_gbps <= 2^20,
+ * 0 <= reconfig_ns, expert_fixed_ns <= 2^40, 0 <= expert_ps_per_token <= 2^30. */
+typedef struct moesched_model {
+  int64_t bytes_per_token;     /* payload of one routed token, bytes            */
+  int64_t link_gbps;           /* port speed in Gb/s == bits per nanosecond     */
+  int64_t reconfig_ns;         /* circuit reconfiguration delay per matching    */
+  int64_t expert_fixed_ns;     /* fixed cost of one expert batch                */
+  int64_t expert_ps_per_token; /* marginal cost per token, picoseconds          */
+} moesched_model_t;
+
+/*
+ * Greedy max-weight decomposition (paper Sec. 3.2: "repeatedly extracts the
+ * maximum-weight perfect matching from the residual matrix and subtracts the
+ * selected matching until all entries become zero").
+ *
+ * Per matrix: R <- D; while k < k_max and R != 0: pi_k <- lexicographically
+ * smallest permutation maximising sum_i R[i][pi(i)] (zero entries are ordinary
+ * weight-0 edges, so pi_k is always a full permutation); d_dur[b][k] <- largest
+ * matched entry (paper Sec. 3.3 / 4.1: the heaviest pair sets the completion
+ * time); the matched entries are served whole and set to zero.
+ *
+ *   d_demand   in   [B][N][N] int32, entries >= 0 and N * max entry <= 2^31-1
+ *   k_max      in   matching budget and output capacity, >= 1
+ *   d_perm     out  [B][k_max][N] uint8
+ *   d_dur      out  [B][k_max] int32
+ *   d_count    out  [B] int32 number of matchings written
+ *   d_residual out  [B][N][N] int32 what is left of D (all zero unless
+ *                   truncated); may be NULL
+ *   d_status   out  [B] int32
+ *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64 work counters, may be NULL:
+ *                   0 shortest-path column scans, 1 augmentations, 2 rows
+ *                   tested for tightness, 3 canonicalisation sweeps that
+ *                   searched, 4 search levels, 5 rotation steps, 6 matchings,
+ *                   7 unused
+ */
+int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
+                          int32_t* d_dur, int32_t* d_count, int32_t* d_residual,
+                          int32_t* d_status, int64_t* d_work, void* stream);
+
+/*
+ * Birkhoff-von Neumann decomposition (paper Sec. 3.1: A = sum_k c_k P_k for a
+ * matrix with equal row and column sums).
+ *
+ * The demand is first made balanced by an exact integer augmentation (the
+ * paper names floating-point Sinkhorn-Knopp scaling as one possible
+ * preprocessing; this library adds padding instead so that everything stays
+ * integral): T = largest row or column sum; the deficits T - rowsum_i and
+ * T - colsum_j are filled by the north-west-corner rule (lowest row first,
+ * then lowest column), giving A = D + E with every row and column summing to
+ * T and at most 2N-1 padded cells. Then, while A != 0 and k < k_max:
+ * pi_k <- lexicographically smallest permutation with A[i][pi(i)] > 0 for all
+ * i; c_k <- min_i A[i][pi_k(i)]; A <- A - c_k P_k. At most N^2 - 2N + 2
+ * matchings result; pass that as k_max for a complete decomposition.
+ *
+ *   d_demand   in   [B][N][N] int32, entries >= 0, every row and column sum
+ *                   <= 2^31-1
+ *   d_perm     out  [B][k_max][N] uint8
+ *   d_coef     out  [B][k_max] int32 coefficients c_k (tokens per pair)
+ *   d_count    out  [B] int32
+ *   d_aug      out  [B][N][N] int32 the balanced matrix A; may be NULL
+ *   d_status   out  [B] int32
+ *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64, may be NULL: 0 augmenting
+ *                   search levels, 1 augmenting-path steps, 2 matchings
+ *                   repaired, 3 canonicalisation sweeps that searched,
+ *                   4 search levels, 5 rotation steps, 6 matchings, 7 rows
+ *                   skipped as unchanged prefix
+ */
+int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
+                           int32_t* d_coef, int32_t* d_count, int32_t* d_aug,
+                           int32_t* d_status, int64_t* d_work, void* stream);
+
+/*
+ * Score a schedule (paper Sec. 4.1: a matching completes after its largest
+ * transfer; "after the dispatch phase of the i-th matching completes, expert
+ * computation begins immediately while communication for the (i+1)-th matching
+ * progresses"; Sec. 3.3: dispatch, compute and combine form a three-machine
+ * flow shop; the "no overlap" panels of Fig. 3 / Fig. 4 run every phase to
+ * completion).
+ *
+ * Per matrix, replaying matchings k = 0 .. count-1 against D:
+ *   served_i = min(dur_k, Dres[i][pi_k(i)]); Dres -= served  (real tokens first)
+ *   g_k = max_i served_i, s_k = sum_i served_i
+ *   t_k    = ceil(dur_k * bytes_per_token * 8 / link_gbps)            [ns]
+ *   comp_k = g_k > 0 ? expert_fixed_ns + ceil(g_k * expert_ps_per_token / 1000) : 0
+ *   Dsp_k = Dsp_{k-1} + reconfig_ns + t_k
+ *   Cmp_k = max(Dsp_k, Cmp_{k-1}) + comp_k
+ *   Cmb_k = max(Cmp_k, Cmb_{k-1}) + reconfig_ns + t_k
+ *   makespan_overlap = Cmb_K;  makespan_serial = sum_k (2 (reconfig_ns + t_k) + comp_k)
+ *   compute_idle = (Cmp_K - Dsp_1) - sum_k comp_k   (0 if K = 0)
+ *   link_idle_tokens = sum_k (N dur_k - s_k);  unserved_tokens = sum Dres
+ *
+ *   d_demand  in   [B][N][N] int32, entries >= 0
+ *   k_stride  in   matchings allocated per matrix in d_perm / d_dur
+ *   d_perm    in   [B][k_stride][N] uint8, each used row a permutation of 0..N-1
+ *   d_dur     in   [B][k_stride] int32, >= 0, sum over k <= 2^40
+ *   d_count   in   [B] int32, 0 <= count <= k_stride
+ *   h_model   in   HOST pointer, read during the call
+ *   d_*       out  [B] int64 each; zero when status is BAD_INPUT
+ *   d_status  out  [B] int32 (OK or BAD_INPUT)
+ */
+int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride,
+                           const uint8_t* d_perm, const int32_t* d_dur, const int32_t* d_count,
+                           const moesched_model_t* h_model, int64_t* d_makespan_overlap_ns,
+                           int64_t* d_makespan_serial_ns, int64_t* d_compute_idle_ns,
+                           int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
+                           int32_t* d_status, void* stream);
+
+/* CUDA error code (cudaError_t as int) of the last failed CUDA call made by
+ * this library on the calling thread; 0 if none. */
+int moesched_last_cuda_error(void);
+
+/* Text for a MOESCHED_* return code or MOESCHED_ST_* status. Never NULL. */
+const char* moesched_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOESCHED_H_ */

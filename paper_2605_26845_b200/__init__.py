@@ -1,0 +1,151 @@
+"""Python binding of libmoesched (argument marshalling only).
+
+Every step of the path -- greedy max-weight decomposition (paper Sec. 3.2),
+Birkhoff-von Neumann decomposition (Sec. 3.1) and schedule scoring (Sec. 4.1) --
+runs in the CUDA kernels behind the C ABI declared in include/moesched.h.
+PyTorch is used for device memory and streams only. There is no CPU fallback:
+a missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from .workload import DEFAULT_MODEL, bvn_capacity  # noqa: F401  (re-exported)
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoesched.so")
+
+ST_OK, ST_TRUNCATED, ST_BAD_INPUT, ST_INTERNAL = 0, 1, -1, -2
+WORK_FIELDS = 8
+MAX_N = 256
+
+
+class MoeschedError(RuntimeError):
+    pass
+
+
+class _Model(ctypes.Structure):
+    _fields_ = [("bytes_per_token", ctypes.c_int64), ("link_gbps", ctypes.c_int64),
+                ("reconfig_ns", ctypes.c_int64), ("expert_fixed_ns", ctypes.c_int64),
+                ("expert_ps_per_token", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen libmoesched.so (built in-tree by paper_2605_26845_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise MoeschedError(f"{LIB_PATH} is missing: run `python -m paper_2605_26845_b200.build` "
+                                "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.moesched_strerror.restype = ctypes.c_char_p
+        for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval",
+                     "moesched_last_cuda_error"):
+            getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        lib = load_library()
+        msg = lib.moesched_strerror(rc).decode()
+        raise MoeschedError(f"{what}: {msg} (rc={rc}, cuda error {lib.moesched_last_cuda_error()})")
+
+
+def _dev(t, dtype, what):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise MoeschedError(f"{what} must be a CUDA tensor (the library has no CPU path)")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise MoeschedError(f"{what} must be contiguous {dtype}")
+    return t
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream(device):
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+@dataclass
+class Schedule:
+    """Ordered matchings of a batch: perm [B, k_max, N] uint8 (perm[b, k, i] = destination of
+    source i), dur [B, k_max] int32 tokens, count [B], status [B]; extra = residual (greedy) or
+    augmented matrix (BvN) if requested; work = per-matrix work counters if requested."""
+    perm: torch.Tensor
+    dur: torch.Tensor
+    count: torch.Tensor
+    status: torch.Tensor
+    extra: torch.Tensor | None = None
+    work: torch.Tensor | None = None
+
+
+def _decompose(fn_name, demand, k_max, want_extra, want_work, out):
+    lib = load_library()
+    demand = _dev(demand, torch.int32, "demand")
+    if demand.dim() != 3 or demand.shape[1] != demand.shape[2]:
+        raise MoeschedError("demand must have shape [B, N, N]")
+    B, N, _ = demand.shape
+    dev = demand.device
+    if out is None:
+        out = Schedule(perm=torch.empty((B, k_max, N), dtype=torch.uint8, device=dev),
+                       dur=torch.empty((B, k_max), dtype=torch.int32, device=dev),
+                       count=torch.empty(B, dtype=torch.int32, device=dev),
+                       status=torch.empty(B, dtype=torch.int32, device=dev),
+                       extra=torch.empty_like(demand) if want_extra else None,
+                       work=torch.empty((B, WORK_FIELDS), dtype=torch.int64, device=dev) if want_work else None)
+    with torch.cuda.device(dev):
+        rc = getattr(lib, fn_name)(B, N, _ptr(demand), int(k_max), _ptr(out.perm), _ptr(out.dur), _ptr(out.count),
+                                   _ptr(out.extra), _ptr(out.status), _ptr(out.work), _stream(dev))
+    _check(rc, fn_name)
+    return out
+
+
+def mw_decompose(demand, k_max, want_residual=False, want_work=False, out=None) -> Schedule:
+    """Greedy max-weight decomposition of every matrix of `demand` [B, N, N] int32 (CUDA)."""
+    return _decompose("moesched_mw_decompose", demand, k_max, want_residual, want_work, out)
+
+
+def bvn_decompose(demand, k_max=None, want_aug=False, want_work=False, out=None) -> Schedule:
+    """Birkhoff-von Neumann decomposition; k_max defaults to N^2 - 2N + 2 (always enough)."""
+    if k_max is None:
+        k_max = bvn_capacity(demand.shape[1])
+    return _decompose("moesched_bvn_decompose", demand, k_max, want_aug, want_work, out)
+
+
+SCORE_FIELDS = ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",
+                "unserved_tokens")
+
+
+def schedule_eval(demand, perm, dur, count, model=None, out=None) -> dict:
+    """Score schedules under the dispatch-compute-combine model. Returns a dict of [B] int64
+    tensors (SCORE_FIELDS) plus 'status' [B] int32; `out` may supply a [5, B] int64 tensor."""
+    lib = load_library()
+    demand = _dev(demand, torch.int32, "demand")
+    perm = _dev(perm, torch.uint8, "perm")
+    dur = _dev(dur, torch.int32, "dur")
+    count = _dev(count, torch.int32, "count")
+    B, N, _ = demand.shape
+    if perm.dim() != 3 or perm.shape[0] != B or perm.shape[2] != N or dur.shape != perm.shape[:2]:
+        raise MoeschedError("perm must be [B, k_stride, N] and dur [B, k_stride]")
+    m = _Model(**{k: int(v) for k, v in (model or DEFAULT_MODEL).items()})
+    dev = demand.device
+    scores = out if out is not None else torch.empty((5, B), dtype=torch.int64, device=dev)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib.moesched_schedule_eval(B, N, _ptr(demand), int(perm.shape[1]), _ptr(perm), _ptr(dur), _ptr(count),
+                                        ctypes.byref(m), _ptr(scores[0]), _ptr(scores[1]), _ptr(scores[2]),
+                                        _ptr(scores[3]), _ptr(scores[4]), _ptr(status), _stream(dev))
+    _check(rc, "moesched_schedule_eval")
+    res = {name: scores[i] for i, name in enumerate(SCORE_FIELDS)}
+    res["status"] = status
+    return res

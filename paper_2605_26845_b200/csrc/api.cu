@@ -1,0 +1,111 @@
+// C ABI of the library: argument checks, launch geometry, error reporting.
+#include "common.cuh"
+
+namespace moesched {
+
+static thread_local int g_last_cuda_error = 0;
+
+// Shared memory one CTA may request on sm_100a (227 KB).
+constexpr size_t SMEM_LIMIT = 227 * 1024;
+
+Geometry plan_geometry(int N) {
+  Geometry ge;
+  ge.cpl = N <= 32 ? 1 : N <= 64 ? 2 : N <= 128 ? 4 : 8;
+  ge.S = (N + ge.cpl - 1) / ge.cpl * ge.cpl;
+  ge.cluster = false;
+  size_t per_warp = warp_smem_bytes(N, ge.S, ge.cpl, false);
+  if (per_warp > SMEM_LIMIT) {
+    ge.cluster = true;
+    per_warp = warp_smem_bytes(N, ge.S, ge.cpl, true);
+  }
+  // several small matrices share a CTA so that an SM can hold up to 64 warps
+  ge.wpb = 1;
+  if (!ge.cluster && N <= 32) ge.wpb = 4;
+  ge.smem = per_warp * ge.wpb;
+  return ge;
+}
+
+static int fail_cuda(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return MOESCHED_ECUDA;
+}
+
+static bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
+static bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7) == 0; }
+
+}  // namespace moesched
+
+using namespace moesched;
+
+extern "C" {
+
+int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm, int32_t* d_dur,
+                          int32_t* d_count, int32_t* d_residual, int32_t* d_status, int64_t* d_work,
+                          void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
+  if (!d_demand || !d_perm || !d_dur || !d_count || !d_status) return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_dur) || !aligned4(d_count) || !aligned4(d_status) ||
+      !aligned4(d_residual) || !aligned8(d_work))
+    return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  cudaError_t e = run_mw(B, N, d_demand, k_max, d_perm, d_dur, d_count, d_residual, d_status,
+                         reinterpret_cast<long long*>(d_work), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm, int32_t* d_coef,
+                           int32_t* d_count, int32_t* d_aug, int32_t* d_status, int64_t* d_work, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
+  if (!d_demand || !d_perm || !d_coef || !d_count || !d_status) return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_coef) || !aligned4(d_count) || !aligned4(d_status) || !aligned4(d_aug) ||
+      !aligned8(d_work))
+    return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  cudaError_t e = run_bvn(B, N, d_demand, k_max, d_perm, d_coef, d_count, d_aug, d_status,
+                          reinterpret_cast<long long*>(d_work), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                           const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                           int64_t* d_makespan_overlap_ns, int64_t* d_makespan_serial_ns,
+                           int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
+                           int32_t* d_status, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_stride < 1) return MOESCHED_EINVAL;
+  if (!d_demand || !d_perm || !d_dur || !d_count || !h_model || !d_makespan_overlap_ns ||
+      !d_makespan_serial_ns || !d_compute_idle_ns || !d_link_idle_tokens || !d_unserved_tokens || !d_status)
+    return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_dur) || !aligned4(d_count) || !aligned4(d_status) ||
+      !aligned8(d_makespan_overlap_ns) || !aligned8(d_makespan_serial_ns) || !aligned8(d_compute_idle_ns) ||
+      !aligned8(d_link_idle_tokens) || !aligned8(d_unserved_tokens))
+    return MOESCHED_EINVAL;
+  const moesched_model_t m = *h_model;
+  const int64_t lim20 = 1LL << 20, lim30 = 1LL << 30, lim40 = 1LL << 40;
+  if (m.bytes_per_token < 1 || m.bytes_per_token > lim20 || m.link_gbps < 1 || m.link_gbps > lim20 ||
+      m.reconfig_ns < 0 || m.reconfig_ns > lim40 || m.expert_fixed_ns < 0 || m.expert_fixed_ns > lim40 ||
+      m.expert_ps_per_token < 0 || m.expert_ps_per_token > lim30)
+    return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  cudaError_t e = run_eval(B, N, d_demand, k_stride, d_perm, d_dur, d_count, m,
+                           reinterpret_cast<long long*>(d_makespan_overlap_ns),
+                           reinterpret_cast<long long*>(d_makespan_serial_ns),
+                           reinterpret_cast<long long*>(d_compute_idle_ns),
+                           reinterpret_cast<long long*>(d_link_idle_tokens),
+                           reinterpret_cast<long long*>(d_unserved_tokens), d_status,
+                           static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* moesched_strerror(int code) {
+  switch (code) {
+    case MOESCHED_OK: return "ok";
+    case MOESCHED_ST_TRUNCATED: return "truncated: the matching budget ran out before the matrix did";
+    case MOESCHED_EINVAL: return "invalid argument, or (as a status) input matrix out of range";
+    case MOESCHED_ECUDA: return "a CUDA call failed, or (as a status) an internal iteration limit was hit";
+    default: return "unknown moesched code";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,293 @@
+// Birkhoff-von Neumann decomposition (paper Sec. 3.1), one warp per demand matrix.
+//
+// The matrix is balanced by north-west-corner padding, then peeled: the support
+// graph (positive entries) is kept as one row-set bit mask per column in
+// registers; after each subtraction only the rows whose matched entry reached
+// zero are re-matched by an augmenting search, and canonicalise() restores the
+// lexicographically smallest perfect matching, starting at the first row whose
+// column changed (earlier rows provably keep theirs).
+#include "common.cuh"
+
+namespace moesched {
+
+// Augmenting search from free row f over alternating paths of the support graph.
+// Returns false when no augmenting path exists (cannot happen for a balanced matrix).
+template <int CPL>
+__device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], int (&mr)[CPL],
+                                             short* x, int& first_changed, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = CPL;
+  unsigned F[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) F[w] = 0u;
+  set_bit<W>(F, f);
+  unsigned visited = 0u;
+  int par[CPL];
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) par[s] = -1;
+  int jf = -1;
+  for (int it = 0; it < N; ++it) {
+    unsigned nxt[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) nxt[w] = 0u;
+    int freeslot = -1;
+#pragma unroll
+    for (int s = CPL - 1; s >= 0; --s) {
+      if (!((visited >> s) & 1u)) {
+        unsigned hit[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) hit[w] = C[s][w] & F[w];
+        if (any_bit<W>(hit)) {
+          visited |= 1u << s;
+          par[s] = lowest_bit<W>(hit);
+          if (mr[s] < 0) freeslot = s;
+          else set_bit<W>(nxt, mr[s]);
+        }
+      }
+    }
+    work[WK_SCAN]++;
+    const unsigned fb = __ballot_sync(FULL, freeslot >= 0);
+    if (fb) {
+      const int L = __ffs(fb) - 1;
+      jf = L * CPL + __shfl_sync(FULL, freeslot, L);
+      break;
+    }
+    bool grew = false;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      F[w] = __reduce_or_sync(FULL, nxt[w]);
+      grew |= F[w] != 0u;
+    }
+    if (!grew) return false;
+  }
+  if (jf < 0) return false;
+  int j = jf;
+  for (int it = 0; it <= N; ++it) {
+    const int L = j / CPL, sl = j % CPL;
+    const int i = __shfl_sync(FULL, pick<CPL>(par, sl), L);
+    const int jprev = x[i];
+    __syncwarp();
+    if (lane == L) put<CPL>(mr, sl, i);
+    if (lane == 0) x[i] = (short)j;
+    __syncwarp();
+    first_changed = min(first_changed, i);
+    work[WK_AUG]++;
+    if (i == f) return true;
+    j = jprev;
+    if (j < 0) return false;
+  }
+  return false;
+}
+
+template <int CPL, bool CLUSTER>
+__global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
+                                                  uint8_t* __restrict__ perm, int32_t* __restrict__ coef,
+                                                  int32_t* __restrict__ count, int32_t* __restrict__ aug,
+                                                  int32_t* __restrict__ status, long long* __restrict__ work_out) {
+  constexpr int W = CPL;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+  if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
+  const int lane = cx.lane, b = cx.b;
+  const MatView A = cx.M;
+  short* x = cx.x;
+  unsigned* hist = cx.hist;
+  const bool loaded = cx.loaded;
+
+  unsigned work[MOESCHED_WORK_FIELDS];
+#pragma unroll
+  for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work[q] = 0u;
+
+  const bool lane_in = lane * CPL < S;
+  int st_code = loaded ? MOESCHED_ST_OK : MOESCHED_ST_INTERNAL;
+  int k = 0;
+
+  // ---- column sums (registers), row sums (one reduction per row), validation ----
+  long long csum[CPL];
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) csum[s] = 0;
+  long long rsum_mine[CPL];   // row sums of the rows lane*CPL+s
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) rsum_mine[s] = 0;
+  int neg = 0;
+  for (int r = 0; r < N; ++r) {
+    long long part = 0;
+    if (lane_in) {
+      RowVec<CPL> rv = load_cols<CPL>(A.row(r), lane);
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        if (lane * CPL + s < N) {
+          neg |= rv.v[s] < 0;
+          csum[s] += rv.v[s];
+          part += rv.v[s];
+        }
+      }
+    }
+    // 64-bit warp sum
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(FULL, part, o);
+    if (lane == r / CPL) put<CPL>(rsum_mine, r % CPL, part);
+  }
+  neg = __any_sync(FULL, neg);
+  long long T = 0;
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) T = max(T, max(csum[s], rsum_mine[s]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) T = max(T, __shfl_xor_sync(FULL, T, o));
+  if (st_code == MOESCHED_ST_OK && (neg || T > 2147483647LL)) st_code = MOESCHED_ST_BAD_INPUT;
+
+  if (st_code == MOESCHED_ST_OK) {
+    // ---- north-west-corner fill of the deficits: lowest row first, then lowest column ----
+    // The staircase visits at most 2N-1 cells; row and column deficits are fetched by shuffle.
+    {
+      int i = 0, j = 0;
+      long long a = 0, bb = 0;
+      bool have_a = false, have_b = false;
+      for (int it = 0; it < 4 * N + 4 && i < N && j < N; ++it) {
+        if (!have_a) { a = T - __shfl_sync(FULL, pick<CPL>(rsum_mine, i % CPL), i / CPL); have_a = true; }
+        if (!have_b) { bb = T - __shfl_sync(FULL, pick<CPL>(csum, j % CPL), j / CPL); have_b = true; }
+        if (a == 0) { ++i; have_a = false; continue; }
+        if (bb == 0) { ++j; have_b = false; continue; }
+        const long long e = min(a, bb);
+        if (lane == 0) A.row(i)[j] += (int)e;
+        a -= e;
+        bb -= e;
+      }
+      __syncwarp();
+    }
+    if (aug != nullptr) {
+      int32_t* ao = aug + (size_t)b * N * N;
+      for (int r = 0; r < N; ++r) {
+        const int* rp = A.row(r);
+        for (int c = lane; c < N; c += 32) ao[(size_t)r * N + c] = rp[c];
+      }
+    }
+
+    // ---- support graph: C[s] = rows with a positive entry in the lane's column s ----
+    unsigned C[CPL][CPL];
+#pragma unroll
+    for (int s = 0; s < CPL; ++s)
+#pragma unroll
+      for (int w = 0; w < W; ++w) C[s][w] = 0u;
+    int nnz = 0;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      for (int q = 0; q < 32; ++q) {
+        const int r = w * 32 + q;
+        if (r >= N) break;
+        if (lane_in) {
+          RowVec<CPL> rv = load_cols<CPL>(A.row(r), lane);
+#pragma unroll
+          for (int s = 0; s < CPL; ++s)
+            if (lane * CPL + s < N && rv.v[s] > 0) { C[s][w] |= 1u << q; ++nnz; }
+        }
+      }
+    }
+    nnz = __reduce_add_sync(FULL, nnz);
+
+    int mr[CPL];
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) mr[s] = -1;
+    for (int r = lane; r < N; r += 32) x[r] = -1;
+    __syncwarp();
+
+    uint8_t* pout = perm + (size_t)b * k_max * N;
+    int32_t* cout_ = coef + (size_t)b * k_max;
+    int first_changed = 0;
+    unsigned freerows[W];   // uniform: rows without a column
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const int lo = w * 32;
+      freerows[w] = N >= lo + 32 ? 0xffffffffu : (N <= lo ? 0u : (0xffffffffu >> (lo + 32 - N)));
+    }
+
+    while (nnz > 0 && k < k_max) {
+      // re-match the free rows
+      bool okm = true;
+      for (int it = 0; it < N; ++it) {
+        const int f = lowest_bit<W>(freerows);
+        if (f < 0) break;
+        first_changed = min(first_changed, f);
+        if (!augment_from<CPL>(N, lane, f, C, mr, x, first_changed, work)) { okm = false; break; }
+        clear_bit<W>(freerows, f);
+      }
+      if (!okm || any_bit<W>(freerows)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      work[WK_SKIP] += first_changed;
+      if (!canonicalise<CPL>(N, lane, first_changed, C, mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+
+      // coefficient = smallest matched entry; subtract it along the matching
+      int val[CPL], cmin = INF32;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        const int c = lane * CPL + s;
+        val[s] = INF32;
+        if (c < N) { val[s] = A.row(mr[s])[c]; cmin = min(cmin, val[s]); }
+      }
+      cmin = __reduce_min_sync(FULL, cmin);
+      first_changed = N;
+      unsigned gone[W];
+#pragma unroll
+      for (int w = 0; w < W; ++w) gone[w] = 0u;
+      int zeroed = 0;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        const int c = lane * CPL + s;
+        if (c < N) {
+          const int nv = val[s] - cmin;
+          A.row(mr[s])[c] = nv;
+          if (nv == 0) {
+            clear_bit<W>(C[s], mr[s]);
+            set_bit<W>(gone, mr[s]);
+            ++zeroed;
+          }
+        }
+      }
+      for (int r = lane; r < N; r += 32) pout[(size_t)k * N + r] = (uint8_t)x[r];
+      if (lane == 0) cout_[k] = cmin;
+      ++k;
+      work[WK_MATCH]++;
+      nnz -= __reduce_add_sync(FULL, zeroed);
+#pragma unroll
+      for (int w = 0; w < W; ++w) freerows[w] = __reduce_or_sync(FULL, gone[w]);
+      // unmatch the rows whose entry vanished
+#pragma unroll
+      for (int s = 0; s < CPL; ++s)
+        if (mr[s] >= 0 && test_bit<W>(freerows, mr[s])) mr[s] = -1;
+      __syncwarp();
+      for (int r = lane; r < N; r += 32)
+        if (test_bit<W>(freerows, r)) x[r] = -1;
+      __syncwarp();
+    }
+    if (st_code == MOESCHED_ST_OK && nnz > 0) st_code = MOESCHED_ST_TRUNCATED;
+  }
+
+  if (st_code == MOESCHED_ST_BAD_INPUT) k = 0;
+  if (lane == 0) {
+    count[b] = k;
+    status[b] = st_code;
+  }
+  if (work_out != nullptr && lane == 0) {
+#pragma unroll
+    for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+  }
+  cluster_epilogue<CLUSTER>();
+}
+
+// ---- host side ---------------------------------------------------------------------------
+
+cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
+                    int32_t* aug, int32_t* status, long long* work, cudaStream_t stream) {
+  const Geometry ge = plan_geometry(N);
+#define MOESCHED_GO(C, CL)                                                                                    \
+  return launch_warp_kernel(bvn_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, count, \
+                            aug, status, work)
+  if (ge.cluster) MOESCHED_GO(8, true);
+  switch (ge.cpl) {
+    case 1: MOESCHED_GO(1, false);
+    case 2: MOESCHED_GO(2, false);
+    case 4: MOESCHED_GO(4, false);
+    default: MOESCHED_GO(8, false);
+  }
+#undef MOESCHED_GO
+}
+
+}  // namespace moesched

@@ -1,0 +1,435 @@
+// Device-side building blocks shared by the three kernels: one warp owns one
+// demand matrix, held in shared memory (for N > 128 spread over the two CTAs of
+// a thread-block cluster), and keeps the matching state in registers.
+//
+// Ownership: lane l owns columns (and rows, where a per-row value is kept in
+// registers) l*CPL .. l*CPL+CPL-1, CPL = 1, 2, 4 or 8, so that a row scan is one
+// vector load per lane. Sets of rows or columns are bit masks of W = CPL 32-bit
+// words; masks that every lane holds identically are "uniform".
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moesched.h"
+
+namespace moesched {
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int INF32 = 0x7fffffff;
+
+enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL = 4, WK_ROT = 5, WK_MATCH = 6, WK_SKIP = 7 };
+
+// ---- small helpers on register arrays -------------------------------------------------
+
+template <int W>
+__device__ __forceinline__ unsigned word_of(const unsigned (&m)[W], int idx) {
+  unsigned w = m[0];
+#pragma unroll
+  for (int k = 1; k < W; ++k)
+    if ((idx >> 5) == k) w = m[k];
+  return w;
+}
+template <int W>
+__device__ __forceinline__ bool test_bit(const unsigned (&m)[W], int idx) {
+  return (word_of<W>(m, idx) >> (idx & 31)) & 1u;
+}
+template <int W>
+__device__ __forceinline__ void set_bit(unsigned (&m)[W], int idx) {
+#pragma unroll
+  for (int k = 0; k < W; ++k)
+    if ((idx >> 5) == k) m[k] |= 1u << (idx & 31);
+}
+template <int W>
+__device__ __forceinline__ void clear_bit(unsigned (&m)[W], int idx) {
+#pragma unroll
+  for (int k = 0; k < W; ++k)
+    if ((idx >> 5) == k) m[k] &= ~(1u << (idx & 31));
+}
+template <int W>
+__device__ __forceinline__ bool any_bit(const unsigned (&m)[W]) {
+  unsigned o = 0;
+#pragma unroll
+  for (int k = 0; k < W; ++k) o |= m[k];
+  return o != 0;
+}
+// lowest set bit of a mask, or -1
+template <int W>
+__device__ __forceinline__ int lowest_bit(const unsigned (&m)[W]) {
+  int r = -1;
+#pragma unroll
+  for (int k = W - 1; k >= 0; --k)
+    if (m[k]) r = k * 32 + __ffs(m[k]) - 1;
+  return r;
+}
+template <int C, typename T>
+__device__ __forceinline__ T pick(const T (&a)[C], int s) {
+  T v = a[0];
+#pragma unroll
+  for (int k = 1; k < C; ++k)
+    if (s == k) v = a[k];
+  return v;
+}
+template <int C, typename T>
+__device__ __forceinline__ void put(T (&a)[C], int s, T v) {
+#pragma unroll
+  for (int k = 0; k < C; ++k)
+    if (s == k) a[k] = v;
+}
+
+// ---- the matrix in shared memory --------------------------------------------------------
+// Rows [0, split) live in this CTA's shared memory, rows [split, N) in the
+// partner CTA of the cluster (far == generic pointer into its shared memory).
+// Without a cluster split >= N and far is unused.
+struct MatView {
+  int* near_;
+  int* far_;
+  int S;      // row stride in ints, a multiple of CPL
+  int split;  // first row held by the partner CTA
+  __device__ __forceinline__ int* row(int r) const {
+    return r < split ? near_ + r * S : far_ + (r - split) * S;
+  }
+};
+
+template <int CPL>
+struct RowVec {
+  int v[CPL];
+};
+
+// Vector load of the lane's CPL consecutive columns of one row. The caller
+// guarantees lane*CPL < S.
+template <int CPL>
+__device__ __forceinline__ RowVec<CPL> load_cols(const int* rowp, int lane) {
+  RowVec<CPL> r;
+  if constexpr (CPL == 1) {
+    r.v[0] = rowp[lane];
+  } else if constexpr (CPL == 2) {
+    int2 t = *reinterpret_cast<const int2*>(rowp + lane * 2);
+    r.v[0] = t.x; r.v[1] = t.y;
+  } else if constexpr (CPL == 4) {
+    int4 t = *reinterpret_cast<const int4*>(rowp + lane * 4);
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+  } else {
+    int4 t = *reinterpret_cast<const int4*>(rowp + lane * 8);
+    int4 q = *reinterpret_cast<const int4*>(rowp + lane * 8 + 4);
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+    r.v[4] = q.x; r.v[5] = q.y; r.v[6] = q.z; r.v[7] = q.w;
+  }
+  return r;
+}
+
+// ---- bulk asynchronous copy global -> shared with an mbarrier ---------------------------
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) {
+  return static_cast<unsigned>(__cvta_generic_to_shared(p));
+}
+
+// Issued by one lane. bytes is a multiple of 16, both addresses 16-byte aligned,
+// bytes < 2^20 (transaction-count range of an mbarrier phase).
+__device__ __forceinline__ void bulk_load_issue(void* smem_dst, const void* gmem_src, unsigned bytes,
+                                                unsigned long long* mbar) {
+  unsigned bar = smem_addr(mbar);
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_addr(smem_dst)),
+      "l"(gmem_src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// All lanes wait for phase 0 of the barrier. The wait is bounded: false means
+// the copy did not land within the limit (never observed; reported, not spun on).
+__device__ __forceinline__ bool bulk_load_wait(unsigned long long* mbar) {
+  unsigned bar = smem_addr(mbar);
+  for (int it = 0; it < (1 << 22); ++it) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+// ---- cluster helpers ---------------------------------------------------------------------
+
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// generic address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ int* map_to_cta(int* local_smem_ptr, unsigned rank) {
+  unsigned long long out;
+  asm volatile("mapa.u64 %0, %1, %2;" : "=l"(out) : "l"((unsigned long long)local_smem_ptr), "r"(rank));
+  return reinterpret_cast<int*>(out);
+}
+
+// ---- load one matrix into shared memory (one warp) ----------------------------------------
+// Copies rows [r0, r1) of the N x N matrix at g into dst with row stride S.
+// Returns false if the bounded wait of the bulk copy ran out.
+__device__ __forceinline__ bool load_rows(int* dst, const int32_t* g, int N, int S, int r0, int r1, int lane,
+                                          unsigned long long* mbar) {
+  const int rows = r1 - r0;
+  if (rows <= 0) return true;
+  const size_t bytes = (size_t)rows * N * 4;
+  const int32_t* src = g + (size_t)r0 * N;
+  const bool bulk = (S == N) && (bytes % 16 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0) &&
+                    bytes < (1u << 20);
+  if (bulk) {
+    if (lane == 0) bulk_load_issue(dst, src, (unsigned)bytes, mbar);
+    __syncwarp();
+    return bulk_load_wait(mbar);
+  }
+  for (int r = 0; r < rows; ++r)
+    for (int c = lane; c < S; c += 32) dst[r * S + c] = c < N ? src[(size_t)r * N + c] : 0;
+  __syncwarp();
+  return true;
+}
+
+// ---- per-warp set-up shared by the kernels ----------------------------------------------------
+// Shared memory of one warp: [matrix rows held here][hist: (N+1)*W words][x: N shorts][mbarrier][flag].
+// In cluster mode the grid has two CTAs (one warp each) per matrix: CTA 0 of the pair
+// works, CTA 1 loads rows [split, N) into its own shared memory and then only keeps
+// them available to CTA 0 (distributed shared memory) until the final cluster barrier.
+struct WarpCtx {
+  int b;          // matrix index
+  int lane;
+  MatView M;
+  unsigned* hist;
+  short* x;
+  bool loaded;    // the matrix arrived in shared memory
+  bool worker;    // false: this warp has nothing more to do (return after cluster_epilogue)
+};
+
+__host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
+__host__ __device__ inline size_t warp_smem_bytes(int N, int S, int W, bool cluster) {
+  const int rows_here = cluster ? (N + 1) / 2 : N;
+  return align16((size_t)rows_here * S * 4) + align16((size_t)(N + 1) * W * 4) + align16((size_t)N * 2) + 16;
+}
+
+template <int CPL, bool CLUSTER>
+__device__ __forceinline__ WarpCtx warp_prologue(int B, int N, int S, const int32_t* demand,
+                                                 unsigned char* smem_raw) {
+  WarpCtx cx;
+  cx.lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int wpb = blockDim.x >> 5;
+  const int split = CLUSTER ? (N + 1) / 2 : N;
+  const int rows_here = CLUSTER ? split : N;
+  const size_t mat_bytes = align16((size_t)rows_here * S * 4);
+  const size_t hist_bytes = align16((size_t)(N + 1) * CPL * 4);
+  const size_t x_bytes = align16((size_t)N * 2);
+  unsigned char* base = smem_raw + (size_t)warp * warp_smem_bytes(N, S, CPL, CLUSTER);
+  int* mat = reinterpret_cast<int*>(base);
+  cx.hist = reinterpret_cast<unsigned*>(base + mat_bytes);
+  cx.x = reinterpret_cast<short*>(base + mat_bytes + hist_bytes);
+  unsigned long long* mbar = reinterpret_cast<unsigned long long*>(base + mat_bytes + hist_bytes + x_bytes);
+  int* peer_flag = reinterpret_cast<int*>(mbar + 1);
+  cx.M.near_ = mat;
+  cx.M.far_ = mat;
+  cx.M.S = S;
+  cx.M.split = split;
+  cx.worker = true;
+  cx.loaded = true;
+  if constexpr (CLUSTER) {
+    const unsigned crank = cluster_ctarank();
+    cx.b = blockIdx.x >> 1;   // grid = 2 B, so always < B
+    const int32_t* g = demand + (size_t)cx.b * N * N;
+    if (crank == 0) cx.loaded = load_rows(mat, g, N, S, 0, split, cx.lane, mbar);
+    else cx.loaded = load_rows(mat, g, N, S, split, N, cx.lane, mbar);
+    if (cx.lane == 0) *peer_flag = cx.loaded ? 1 : 0;
+    cx.M.far_ = map_to_cta(mat, 1);
+    cluster_sync_all();
+    if (crank != 0) cx.worker = false;
+    else cx.loaded = cx.loaded && (*map_to_cta(peer_flag, 1) != 0);
+  } else {
+    cx.b = blockIdx.x * wpb + warp;
+    if (cx.b >= B) { cx.worker = false; return cx; }
+    cx.loaded = load_rows(mat, demand + (size_t)cx.b * N * N, N, S, 0, N, cx.lane, mbar);
+  }
+  return cx;
+}
+
+// Every warp of a cluster launch passes here exactly once before it returns.
+template <bool CLUSTER>
+__device__ __forceinline__ void cluster_epilogue() {
+  if constexpr (CLUSTER) cluster_sync_all();
+}
+
+// ---- lexicographically smallest perfect matching -------------------------------------------
+//
+// State: C[s] = set of rows adjacent to the lane's column s in the graph (tight
+// edges for the greedy step, positive entries for Birkhoff), mr[s] = row matched
+// to that column, x[r] = column matched to row r (shared memory, one entry per
+// row). On entry (mr, x) is some perfect matching of the graph that already
+// agrees with the answer on rows < start. For each row i >= start in order the
+// routine finds the lowest column that row i can take in a perfect matching that
+// keeps rows < i fixed: an edge (i, j) outside the matching is usable iff row
+// mr[j] reaches row i along alternating steps r -> r' (r adjacent to the column
+// of r') among the rows not yet fixed; the matching is then rotated along that
+// cycle. hist holds one row set per search level to retrace the cycle.
+template <int CPL>
+__device__ __forceinline__ bool canonicalise(int N, int lane, int start, const unsigned (&C)[CPL][CPL],
+                                             int (&mr)[CPL], short* x, unsigned* hist,
+                                             unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = CPL;
+  bool ok_all = true;
+  unsigned alive[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    int lo = w * 32, hi = lo + 32;
+    unsigned m = 0xffffffffu;
+    if (start > lo) m = start >= hi ? 0u : (0xffffffffu << (start - lo));
+    if (N < hi) m &= N <= lo ? 0u : (0xffffffffu >> (hi - N));
+    alive[w] = m;
+  }
+  for (int i = start; i < N; ++i) {
+    const int xi = x[i];
+    // columns below the current one that row i is adjacent to and whose row is still free to move
+    bool cand = false;
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) {
+      int c = lane * CPL + s;
+      cand |= (c < xi) && test_bit<W>(C[s], i) && (mr[s] > i);
+    }
+    if (__ballot_sync(FULL, cand) == 0u) {
+      clear_bit<W>(alive, i);
+      continue;
+    }
+    work[WK_SWEEP]++;
+    // backward search from row i
+    unsigned anc[W], F[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) anc[w] = F[w] = 0u;
+    set_bit<W>(anc, i);
+    set_bit<W>(F, i);
+    int level = 0;
+    if (lane < W) hist[lane] = pick<W>(F, lane);
+    for (int it = 0; it < N; ++it) {
+      unsigned acc[W];
+#pragma unroll
+      for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        if (mr[s] >= 0 && test_bit<W>(F, mr[s])) {
+#pragma unroll
+          for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
+        }
+      }
+      bool grew = false;
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        unsigned a = __reduce_or_sync(FULL, acc[w]) & alive[w] & ~anc[w];
+        anc[w] |= a;
+        F[w] = a;
+        grew |= a != 0u;
+      }
+      work[WK_LEVEL]++;
+      if (!grew) break;
+      ++level;
+      if (lane < W) hist[level * W + lane] = pick<W>(F, lane);
+    }
+    __syncwarp();
+    // lowest column row i may take
+    int myslot = -1;
+#pragma unroll
+    for (int s = CPL - 1; s >= 0; --s)
+      if (mr[s] >= 0 && test_bit<W>(C[s], i) && test_bit<W>(anc, mr[s])) myslot = s;
+    unsigned ball = __ballot_sync(FULL, myslot >= 0);
+    if (ball == 0u) { ok_all = false; clear_bit<W>(alive, i); continue; }   // cannot happen: column xi qualifies
+    const int L = __ffs(ball) - 1;
+    const int sl = __shfl_sync(FULL, myslot, L);
+    const int jstar = L * CPL + sl;
+    if (jstar != xi) {
+      int cur = __shfl_sync(FULL, pick<CPL>(mr, sl), L);   // row that gives up column jstar
+      // level at which that row was reached
+      int lvl = 0;
+      for (int d = 1; d <= level; ++d) {
+        unsigned hw = hist[d * W + (cur >> 5)];
+        if ((hw >> (cur & 31)) & 1u) lvl = d;
+      }
+      if (lvl == 0) ok_all = false;
+      // walk towards row i: each row takes the column of its successor on the cycle
+      while (lvl > 0) {
+        unsigned Hm[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) Hm[w] = hist[(lvl - 1) * W + w];
+        int ms = -1;
+#pragma unroll
+        for (int s = CPL - 1; s >= 0; --s)
+          if (mr[s] >= 0 && test_bit<W>(Hm, mr[s]) && test_bit<W>(C[s], cur)) ms = s;
+        unsigned b2 = __ballot_sync(FULL, ms >= 0);
+        if (b2 == 0u) { ok_all = false; break; }
+        const int L2 = __ffs(b2) - 1;
+        const int s2 = __shfl_sync(FULL, ms, L2);
+        const int nxt = __shfl_sync(FULL, pick<CPL>(mr, s2), L2);
+        if (lane == L2) put<CPL>(mr, s2, cur);
+        if (lane == 0) x[cur] = (short)(L2 * CPL + s2);
+        cur = nxt;
+        --lvl;
+        work[WK_ROT]++;
+      }
+      if (lane == L) put<CPL>(mr, sl, i);
+      if (lane == 0) x[i] = (short)jstar;
+      __syncwarp();
+    }
+    clear_bit<W>(alive, i);
+  }
+  return ok_all;
+}
+
+// ---- host-side launch geometry ---------------------------------------------------------------
+struct Geometry {
+  int cpl;       // columns per lane: 1, 2, 4 or 8
+  int S;         // shared-memory row stride in ints
+  bool cluster;  // matrix split over a 2-CTA cluster
+  int wpb;       // warps (matrices) per CTA
+  size_t smem;   // dynamic shared memory per CTA
+};
+Geometry plan_geometry(int N);
+
+cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
+                   int32_t* residual, int32_t* status, long long* work, cudaStream_t stream);
+cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
+                    int32_t* aug, int32_t* status, long long* work, cudaStream_t stream);
+cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
+                     const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
+                     long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
+                     cudaStream_t stream);
+
+// Launch helper shared by the three kernels.
+template <typename Kernel, typename... Args>
+cudaError_t launch_warp_kernel(Kernel kern, const Geometry& ge, int B, cudaStream_t stream, Args... args) {
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ge.smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(32 * ge.wpb);
+  cfg.dynamicSmemBytes = ge.smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (ge.cluster) {
+    cfg.gridDim = dim3(2 * B);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  } else {
+    cfg.gridDim = dim3((B + ge.wpb - 1) / ge.wpb);
+  }
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+}  // namespace moesched

@@ -1,0 +1,155 @@
+// Schedule scoring (paper Sec. 4.1 "Execution time", Sec. 3.3), one warp per matrix.
+//
+// The demand matrix sits in shared memory and is consumed as the matchings are
+// replayed; the schedule streams in from global memory. Matching k serves
+// min(dur_k, remaining demand) tokens on each pair; the busiest pair drives the
+// expert batch time; dispatch, compute and combine advance as a three-stage
+// pipeline. Link idleness is obtained from totals: sum_k (N dur_k - s_k) equals
+// N * sum_k dur_k minus all served tokens.
+#include "common.cuh"
+
+namespace moesched {
+
+__device__ __forceinline__ long long warp_sum64(long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+  return v;
+}
+
+template <int CPL>
+__device__ __forceinline__ long long matrix_sum(const MatView& M, int N, int lane, bool lane_in, int* any_negative) {
+  long long acc = 0;
+  int neg = 0;
+  for (int r = 0; r < N; ++r) {
+    if (lane_in) {
+      RowVec<CPL> rv = load_cols<CPL>(M.row(r), lane);
+#pragma unroll
+      for (int s = 0; s < CPL; ++s)
+        if (lane * CPL + s < N) { acc += rv.v[s]; neg |= rv.v[s] < 0; }
+    }
+  }
+  if (any_negative) *any_negative = __any_sync(FULL, neg);
+  return warp_sum64(acc);
+}
+
+template <int CPL, bool CLUSTER>
+__global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_stride,
+                                                   const uint8_t* __restrict__ perm, const int32_t* __restrict__ dur,
+                                                   const int32_t* __restrict__ count, moesched_model_t model,
+                                                   long long* __restrict__ overlap, long long* __restrict__ serial,
+                                                   long long* __restrict__ idle_ns, long long* __restrict__ idle_tok,
+                                                   long long* __restrict__ unserved, int32_t* __restrict__ status) {
+  constexpr int W = CPL;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+  if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
+  const int lane = cx.lane, b = cx.b;
+  const MatView D = cx.M;
+  const bool lane_in = lane * CPL < S;
+
+  int bad = cx.loaded ? 0 : 1;
+  int neg = 0;
+  const long long total = matrix_sum<CPL>(D, N, lane, lane_in, &neg);
+  bad |= neg;
+  const int K = count[b];
+  if (K < 0 || K > k_stride) bad = 1;
+
+  long long dsp = 0, cmp = 0, cmb = 0, ser = 0, comp_sum = 0, dsp1 = 0, dur_sum = 0;
+  const uint8_t* pb = perm + (size_t)b * k_stride * N;
+  const int32_t* db = dur + (size_t)b * k_stride;
+
+  if (!bad) {
+    for (int k0 = 0; k0 < K && !bad; k0 += 32) {
+      // lane q prepares the transfer time of matching k0+q
+      const int kk = k0 + lane;
+      const int dk_mine = kk < K ? db[kk] : 0;
+      if (__any_sync(FULL, dk_mine < 0)) { bad = 1; break; }
+      const long long t_mine =
+          ((long long)dk_mine * model.bytes_per_token * 8 + model.link_gbps - 1) / model.link_gbps;
+      const int kend = min(32, K - k0);
+      for (int q = 0; q < kend; ++q) {
+        const int dk = __shfl_sync(FULL, dk_mine, q);
+        const long long t = __shfl_sync(FULL, t_mine, q);
+        const uint8_t* pk = pb + (size_t)(k0 + q) * N;
+        unsigned cols[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) cols[w] = 0u;
+        int g = 0, oob = 0;
+#pragma unroll
+        for (int s = 0; s < CPL; ++s) {
+          const int r = lane * CPL + s;
+          if (r < N) {
+            const int j = pk[r];
+            if (j < N) {
+              set_bit<W>(cols, j);
+              int* p = D.row(r) + j;
+              const int val = *p;
+              const int sv = min(dk, val);
+              *p = val - sv;
+              g = max(g, sv);
+            } else {
+              oob = 1;
+            }
+          }
+        }
+        int seen = 0;
+#pragma unroll
+        for (int w = 0; w < W; ++w) seen += __popc(__reduce_or_sync(FULL, cols[w]));
+        if (__any_sync(FULL, oob) || seen != N) { bad = 1; break; }
+        g = __reduce_max_sync(FULL, g);
+        const long long comp =
+            g > 0 ? model.expert_fixed_ns + ((long long)g * model.expert_ps_per_token + 999) / 1000 : 0;
+        const long long leg = model.reconfig_ns + t;
+        dsp += leg;
+        if (k0 + q == 0) dsp1 = dsp;
+        cmp = max(dsp, cmp) + comp;
+        cmb = max(cmp, cmb) + leg;
+        ser += 2 * leg + comp;
+        comp_sum += comp;
+        dur_sum += dk;
+        __syncwarp();
+      }
+    }
+    if (dur_sum > (1LL << 40)) bad = 1;
+  }
+
+  long long left = 0;
+  if (!bad) {
+    __syncwarp();
+    left = matrix_sum<CPL>(D, N, lane, lane_in, nullptr);
+  }
+  if (lane == 0) {
+    if (bad) {
+      overlap[b] = serial[b] = idle_ns[b] = idle_tok[b] = unserved[b] = 0;
+      status[b] = MOESCHED_ST_BAD_INPUT;
+    } else {
+      overlap[b] = cmb;
+      serial[b] = ser;
+      idle_ns[b] = K > 0 ? (cmp - dsp1) - comp_sum : 0;
+      idle_tok[b] = (long long)N * dur_sum - (total - left);
+      unserved[b] = left;
+      status[b] = MOESCHED_ST_OK;
+    }
+  }
+  cluster_epilogue<CLUSTER>();
+}
+
+cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
+                     const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
+                     long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
+                     cudaStream_t stream) {
+  const Geometry ge = plan_geometry(N);
+#define MOESCHED_GO(C, CL)                                                                                       \
+  return launch_warp_kernel(eval_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, count, \
+                            model, overlap, serial, idle_ns, idle_tok, unserved, status)
+  if (ge.cluster) MOESCHED_GO(8, true);
+  switch (ge.cpl) {
+    case 1: MOESCHED_GO(1, false);
+    case 2: MOESCHED_GO(2, false);
+    case 4: MOESCHED_GO(4, false);
+    default: MOESCHED_GO(8, false);
+  }
+#undef MOESCHED_GO
+}
+
+}  // namespace moesched

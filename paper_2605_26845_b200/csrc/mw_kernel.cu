@@ -1,0 +1,234 @@
+// Greedy max-weight decomposition (paper Sec. 3.2), one warp per demand matrix.
+//
+// Each greedy step solves one assignment problem on the residual matrix R by
+// shortest augmenting paths on cost = -R (a Jonker-Volgenant style search that
+// keeps only the column duals v and settles one column per scan), derives the
+// row duals, marks the tight edges and hands that graph to canonicalise(), which
+// returns the lexicographically smallest optimal permutation. The matched
+// entries are then served whole; the largest one is the matching's duration.
+#include "common.cuh"
+
+namespace moesched {
+
+template <int CPL>
+struct MwState {
+  int v[CPL];     // column duals of the cost problem
+  int mr[CPL];    // row assigned to the lane's column, -1 if free
+};
+
+// One assignment problem from scratch. Returns false if an iteration limit was hit.
+template <int CPL>
+__device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int lane, bool lane_in,
+                                                 MwState<CPL>& st, short* x, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  bool ok = true;
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) { st.v[s] = 0; st.mr[s] = -1; }
+  for (int r = lane; r < N; r += 32) x[r] = -1;
+  __syncwarp();
+  for (int f = 0; f < N; ++f) {
+    int dist[CPL], pred[CPL];
+    unsigned scanned = 0u;     // bit s: the lane's column s is settled
+    {
+      RowVec<CPL> rv;
+      if (lane_in) rv = load_cols<CPL>(R.row(f), lane);
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        bool valid = lane * CPL + s < N;
+        dist[s] = valid ? -rv.v[s] - st.v[s] : INF32;
+        pred[s] = f;
+        if (!valid) scanned |= 1u << s;
+      }
+    }
+    int jfin = -1, mu = 0;
+    for (int it = 0; it < N; ++it) {
+      int lmin = INF32, lslot = 0;
+#pragma unroll
+      for (int s = CPL - 1; s >= 0; --s) {
+        int d = ((scanned >> s) & 1u) ? INF32 : dist[s];
+        if (d <= lmin) { lmin = d; lslot = s; }
+      }
+      mu = __reduce_min_sync(FULL, lmin);
+      const unsigned ball = __ballot_sync(FULL, lmin == mu);
+      const int L = __ffs(ball) - 1;
+      const int sl = __shfl_sync(FULL, lslot, L);
+      if (lane == L) scanned |= 1u << sl;
+      const int i = __shfl_sync(FULL, pick<CPL>(st.mr, sl), L);
+      work[WK_SCAN]++;
+      if (i < 0) { jfin = L * CPL + sl; break; }
+      const int vj = __shfl_sync(FULL, pick<CPL>(st.v, sl), L);
+      RowVec<CPL> rv;
+      if (lane_in) rv = load_cols<CPL>(R.row(i), lane);
+      const int rij = __shfl_sync(FULL, pick<CPL>(rv.v, sl), L);
+      const int h = -rij - vj - mu;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        int nd = -rv.v[s] - st.v[s] - h;
+        if (!((scanned >> s) & 1u) && nd < dist[s]) { dist[s] = nd; pred[s] = i; }
+      }
+    }
+    if (jfin < 0) { ok = false; break; }
+    // settled columns move their dual so that the new shortest-path tree stays tight
+#pragma unroll
+    for (int s = 0; s < CPL; ++s)
+      if (((scanned >> s) & 1u) && lane * CPL + s < N) st.v[s] += dist[s] - mu;
+    // flip the path back to row f
+    int j = jfin;
+    for (int it = 0; it <= N; ++it) {
+      const int L = j / CPL, sl = j % CPL;
+      const int i = __shfl_sync(FULL, pick<CPL>(pred, sl), L);
+      const int jprev = x[i];
+      __syncwarp();
+      if (lane == L) put<CPL>(st.mr, sl, i);
+      if (lane == 0) x[i] = (short)j;
+      __syncwarp();
+      if (i == f) break;
+      j = jprev;
+      if (j < 0) { ok = false; break; }
+    }
+    work[WK_AUG]++;
+  }
+  return ok;
+}
+
+template <int CPL, bool CLUSTER>
+__global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
+                                                 uint8_t* __restrict__ perm, int32_t* __restrict__ dur,
+                                                 int32_t* __restrict__ count, int32_t* __restrict__ residual,
+                                                 int32_t* __restrict__ status, long long* __restrict__ work_out) {
+  constexpr int W = CPL;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+  if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
+  const int lane = cx.lane, b = cx.b;
+  const MatView R = cx.M;
+  short* x = cx.x;
+  unsigned* hist = cx.hist;
+  const bool loaded = cx.loaded;
+
+  unsigned work[MOESCHED_WORK_FIELDS];
+#pragma unroll
+  for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work[q] = 0u;
+
+  const bool lane_in = lane * CPL < S;
+  int st_code = MOESCHED_ST_OK;
+  int k = 0;
+
+  // validate, find the largest entry, count the non-zero entries
+  int nnz = 0;
+  {
+    int mx = 0, neg = 0, cnt = 0;
+    for (int r = 0; r < N; ++r) {
+      if (lane_in) {
+        RowVec<CPL> rv = load_cols<CPL>(R.row(r), lane);
+#pragma unroll
+        for (int s = 0; s < CPL; ++s) {
+          if (lane * CPL + s < N) {
+            neg |= rv.v[s] < 0;
+            mx = max(mx, rv.v[s]);
+            cnt += rv.v[s] != 0;
+          }
+        }
+      }
+    }
+    neg = __any_sync(FULL, neg);
+    mx = __reduce_max_sync(FULL, mx);
+    nnz = __reduce_add_sync(FULL, cnt);
+    if (neg || (long long)mx * N > 2147483647LL) st_code = MOESCHED_ST_BAD_INPUT;
+    if (!loaded) st_code = MOESCHED_ST_INTERNAL;
+  }
+
+  if (st_code == MOESCHED_ST_OK) {
+    MwState<CPL> st;
+    uint8_t* pout = perm + (size_t)b * k_max * N;
+    int32_t* dout = dur + (size_t)b * k_max;
+    while (k < k_max && nnz > 0) {
+      if (!solve_assignment<CPL>(R, N, lane, lane_in, st, x, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      // tight edges: row r is tight to column c iff cost(r,c) - v[c] equals the row minimum
+      unsigned C[CPL][CPL];
+#pragma unroll
+      for (int s = 0; s < CPL; ++s)
+#pragma unroll
+        for (int w = 0; w < W; ++w) C[s][w] = 0u;
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        for (int q = 0; q < 32; ++q) {
+          const int r = w * 32 + q;
+          if (r >= N) break;
+          RowVec<CPL> rv;
+          if (lane_in) rv = load_cols<CPL>(R.row(r), lane);
+          int red[CPL], lm = INF32;
+#pragma unroll
+          for (int s = 0; s < CPL; ++s) {
+            red[s] = (lane * CPL + s < N) ? -rv.v[s] - st.v[s] : INF32;
+            lm = min(lm, red[s]);
+          }
+          const int u = __reduce_min_sync(FULL, lm);
+#pragma unroll
+          for (int s = 0; s < CPL; ++s)
+            if (red[s] == u && lane * CPL + s < N) C[s][w] |= 1u << q;
+        }
+      }
+      work[WK_TIGHT] += N;
+      if (!canonicalise<CPL>(N, lane, 0, C, st.mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      // serve: the heaviest matched pair sets the duration; matched entries are sent whole
+      int dmax = 0, served = 0;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        const int c = lane * CPL + s;
+        if (c < N && st.mr[s] >= 0) {
+          int* p = R.row(st.mr[s]) + c;
+          const int val = *p;
+          dmax = max(dmax, val);
+          served += val != 0;
+          *p = 0;
+        }
+      }
+      dmax = __reduce_max_sync(FULL, dmax);
+      nnz -= __reduce_add_sync(FULL, served);
+      __syncwarp();
+      for (int r = lane; r < N; r += 32) pout[(size_t)k * N + r] = (uint8_t)x[r];
+      if (lane == 0) dout[k] = dmax;
+      ++k;
+      work[WK_MATCH]++;
+    }
+    if (st_code == MOESCHED_ST_OK && nnz > 0) st_code = MOESCHED_ST_TRUNCATED;
+  }
+
+  if (st_code == MOESCHED_ST_BAD_INPUT) k = 0;
+  if (lane == 0) {
+    count[b] = k;
+    status[b] = st_code;
+  }
+  if (residual != nullptr && st_code != MOESCHED_ST_BAD_INPUT) {
+    int32_t* ro = residual + (size_t)b * N * N;
+    for (int r = 0; r < N; ++r) {
+      const int* rp = R.row(r);
+      for (int c = lane; c < N; c += 32) ro[(size_t)r * N + c] = rp[c];
+    }
+  }
+  if (work_out != nullptr && lane == 0) {
+#pragma unroll
+    for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+  }
+  cluster_epilogue<CLUSTER>();
+}
+
+// ---- host side ---------------------------------------------------------------------------
+
+cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
+                   int32_t* residual, int32_t* status, long long* work, cudaStream_t stream) {
+  const Geometry ge = plan_geometry(N);
+#define MOESCHED_GO(C, CL)                                                                                  \
+  return launch_warp_kernel(mw_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur, count, \
+                            residual, status, work)
+  if (ge.cluster) MOESCHED_GO(8, true);
+  switch (ge.cpl) {
+    case 1: MOESCHED_GO(1, false);
+    case 2: MOESCHED_GO(2, false);
+    case 4: MOESCHED_GO(4, false);
+    default: MOESCHED_GO(8, false);
+  }
+#undef MOESCHED_GO
+}
+
+}  // namespace moesched

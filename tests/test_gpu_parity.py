@@ -1,0 +1,140 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_26845_b200 as ms
+from paper_2605_26845_b200.workload import (CONFIGS, DEFAULT_MODEL, bvn_capacity, make_demand,
+                                            random_matrices, structured_cases)
+
+pytestmark = pytest.mark.gpu
+
+KINDS = [dict(kind="uniform", high=1000), dict(kind="ties"), dict(kind="uniform", high=9, zero_frac=0.6)]
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def assert_schedule_equal(gpu, ref, key):
+    """perm / dur are compared on the first count[b] matchings only (the rest is unspecified)."""
+    count = gpu.count.cpu().numpy()
+    status = gpu.status.cpu().numpy()
+    assert (status == ref["status"]).all(), (status, ref["status"])
+    assert (count == ref["count"]).all(), (count, ref["count"])
+    perm = gpu.perm.cpu().numpy()
+    dur = gpu.dur.cpu().numpy()
+    kk = np.arange(perm.shape[1])[None, :] < count[:, None]
+    assert (perm[kk] == ref["perm"][kk]).all()
+    assert (dur[kk] == ref[key][kk]).all()
+
+
+def check_all(D, k_mw, k_bvn, model=DEFAULT_MODEL, threads=8):
+    d = dev(D)
+    g = ms.mw_decompose(d, k_mw, want_residual=True)
+    rg = oracle.mw_decompose(D, k_mw, threads=threads)
+    assert_schedule_equal(g, rg, "dur")
+    ok = rg["status"] >= 0
+    assert (g.extra.cpu().numpy()[ok] == rg["residual"][ok]).all()
+    v = ms.bvn_decompose(d, k_bvn, want_aug=True)
+    rv = oracle.bvn_decompose(D, k_bvn, threads=threads)
+    assert_schedule_equal(v, rv, "coef")
+    ok = rv["status"] >= 0
+    assert (v.extra.cpu().numpy()[ok] == rv["aug"][ok]).all()
+    for sched, ref, key in ((g, rg, "dur"), (v, rv, "coef")):
+        good = dev(ref["status"] >= 0)
+        count = torch.where(good, sched.count, torch.zeros_like(sched.count))
+        # rows beyond count are never read, so uninitialised memory there is fine
+        s = ms.schedule_eval(d, sched.perm, sched.dur, count, model)
+        cnt = np.where(ref["status"] >= 0, ref["count"], 0).astype(np.int32)
+        rs = oracle.schedule_eval(D, ref["perm"], ref[key], cnt, model, threads=threads)
+        for name in ms.SCORE_FIELDS + ("status",):
+            assert (s[name].cpu().numpy() == rs[name]).all(), name
+    return g, v
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 13, 17, 31, 32, 33, 48, 64])
+@pytest.mark.parametrize("kw", KINDS)
+def test_small_matrices_full_decompositions(N, kw):
+    D = random_matrices(5, N, seed=1000 + N, **kw)
+    check_all(D, N * N + 1, bvn_capacity(N))
+
+
+@pytest.mark.parametrize("N", [65, 96, 100, 128, 129, 192, 232, 233, 256])
+@pytest.mark.parametrize("kw", KINDS)
+def test_large_matrices_prefix(N, kw):
+    """The oracle needs O(N^3) per matching, so large sizes are compared on a schedule prefix."""
+    D = random_matrices(3, N, seed=2000 + N, **kw)
+    check_all(D, 6, 10)
+
+
+@pytest.mark.parametrize("N", [1, 2, 5, 8, 17, 64, 100])
+def test_closed_form_cases(N):
+    cases = structured_cases(N, m=7)
+    D = np.stack(list(cases.values()))
+    g, v = check_all(D, N + 2, N + 2)
+    names = list(cases)
+    gc = g.count.cpu().numpy()
+    vc = v.count.cpu().numpy()
+    assert gc[names.index("zero")] == 0 and vc[names.index("zero")] == 0
+    assert gc[names.index("scaled_permutation")] == 1 and vc[names.index("scaled_permutation")] == 1
+    assert gc[names.index("uniform")] == N and vc[names.index("uniform")] == N
+    assert gc[names.index("hot_column")] == N and gc[names.index("diagonal")] == 1
+
+
+def test_bad_inputs_and_budget():
+    D = make_demand(1, 6)
+    D[1, 2, 3] = -1
+    D[4, 0, 0] = 2**31 - 1          # N * max entry and the row sum overflow 31 bits
+    check_all(D, 8, 50)
+    check_all(D, 1, 1)
+    check_all(D, 3, 7)
+
+
+def test_eval_rejects_bad_schedules():
+    D = make_demand(1, 4)
+    d = dev(D)
+    g = ms.mw_decompose(d, 8)
+    perm = g.perm.cpu().numpy().copy()
+    dur = g.dur.cpu().numpy().copy()
+    count = g.count.cpu().numpy().copy()
+    perm[0, 1, 3] = perm[0, 1, 2]   # repeated column
+    perm[1, 0, 0] = 200             # out of range
+    dur[2, 0] = -4
+    count[3] = 9                    # beyond the stride
+    s = ms.schedule_eval(d, dev(perm), dev(dur), dev(count))
+    r = oracle.schedule_eval(D, perm, dur, count, DEFAULT_MODEL)
+    assert list(r["status"]) == [-1, -1, -1, -1]
+    for name in ms.SCORE_FIELDS + ("status",):
+        assert (s[name].cpu().numpy() == r[name]).all(), name
+
+
+def test_argument_errors_are_reported():
+    d = dev(make_demand(1, 2))
+    with pytest.raises(ms.MoeschedError):
+        ms.mw_decompose(d, 0)
+    with pytest.raises(ms.MoeschedError):
+        ms.mw_decompose(d.cpu(), 8)
+    with pytest.raises(ms.MoeschedError):
+        ms.schedule_eval(d, torch.zeros((2, 1, 8), dtype=torch.uint8, device="cuda"),
+                         torch.zeros((2, 1), dtype=torch.int32, device="cuda"),
+                         torch.zeros(2, dtype=torch.int32, device="cuda"), dict(DEFAULT_MODEL, link_gbps=0))
+    too_big = torch.zeros((1, 257, 257), dtype=torch.int32, device="cuda")
+    with pytest.raises(ms.MoeschedError):
+        ms.mw_decompose(too_big, 4)
+
+
+def test_runs_are_deterministic_and_stream_ordered():
+    D = make_demand(2, 64)
+    d = dev(D)
+    a = ms.bvn_decompose(d)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b = ms.bvn_decompose(d)
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert (a.count == b.count).all() and (a.status == b.status).all()
+    kk = (torch.arange(a.perm.shape[1], device="cuda")[None, :] < a.count[:, None])
+    assert (a.perm[kk] == b.perm[kk]).all() and (a.dur[kk] == b.dur[kk]).all()
