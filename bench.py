@@ -1,0 +1,327 @@
+"""Benchmark: demand-matrix decompositions per second on the headline workload.
+
+One step = one pass of the whole path over one batch of B demand matrices:
+greedy max-weight decomposition (k_max = 64), Birkhoff-von Neumann decomposition
+(capacity N^2-2N+2) and the scoring of both schedules -- four kernel launches.
+A "decomposition" is one demand matrix taken through all of it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched through torch.distributed.run) every rank processes its own
+B matrices; there is no exchange step, so no collective touches the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2605_26845_b200.workload import CONFIGS, DEFAULT_MODEL, bvn_capacity, make_demand  # noqa: E402
+
+METRIC = "demand-matrix decompositions/sec at N=64 (greedy+BvN)"
+UNIT = "decompositions/s"
+CFG = 3
+K_MW = 64
+FALLBACK_HBM_GBS = 6650.0
+# Issue-rate ceiling for plain integer work: 148 SMs x 4 warp schedulers x 32 lanes, one
+# instruction per scheduler per clock, at the SM clock sampled during the run.
+ALU_LANES_PER_CLK = 148 * 4 * 32
+
+
+def workload_name(B):
+    c = CONFIGS[CFG]
+    return (f"config 3: N={c['N']}, B={B}, {c['tokens']} tokens/rank, {c['experts']} experts top-{c['top_k']}, "
+            f"Zipf s={c['s']} reshuffled per matrix; greedy k_max={K_MW} + BvN (capacity "
+            f"{bvn_capacity(c['N'])}), both scored")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def __enter__(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v == "Active":
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def algorithmic_ops(work_mw, work_bvn, N):
+    """Integer lane-operations the method itself needs, from the kernels' work counters
+    (per column or row touched: a handful of adds / compares / bit operations)."""
+    W = (N + 31) // 32
+    mw = (6 * N * work_mw[:, 0] + 4 * work_mw[:, 1] + 4 * N * work_mw[:, 2] + 4 * N * W * work_mw[:, 4]
+          + 6 * N * work_mw[:, 5] + 4 * N * work_mw[:, 6] + 4 * N * work_mw[:, 3])
+    bvn = (4 * N * W * work_bvn[:, 0] + 4 * work_bvn[:, 1] + 4 * N * W * work_bvn[:, 4] + 6 * N * work_bvn[:, 5]
+           + 6 * N * work_bvn[:, 6] + 4 * N * work_bvn[:, 3])
+    return float(mw.sum()), float(bvn.sum())
+
+
+def oracle_rate(D, threads, k_bvn):
+    """Whole path on the CPU checker: matrices per second (wall clock)."""
+    import oracle
+    t0 = time.perf_counter()
+    g = oracle.mw_decompose(D, K_MW, threads=threads, want_residual=False)
+    v = oracle.bvn_decompose(D, k_bvn, threads=threads, want_aug=False)
+    oracle.schedule_eval(D, g["perm"], g["dur"], g["count"], DEFAULT_MODEL, threads=threads)
+    oracle.schedule_eval(D, v["perm"], v["coef"], v["count"], DEFAULT_MODEL, threads=threads)
+    return D.shape[0] / (time.perf_counter() - t0)
+
+
+def run_reference(args, rank):
+    """The CPU checker as it stands, on the host cores, a bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    threads = oracle.hardware_threads()
+    sample = max(threads, 16)
+    N = CONFIGS[CFG]["N"]
+    D = make_demand(CFG, sample)
+    cap = bvn_capacity(N)
+    for _ in range(args.warmup):
+        oracle_rate(D[:threads], threads, cap)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_rate(D, threads, cap)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    what = f"first {sample} matrices of the workload per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": workload_name(CONFIGS[CFG]["B"]), "sample": what},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=None, help="matrices per GPU (default: the configuration's B)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2605_26845_b200 as ms
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    ms.load_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg = CONFIGS[CFG]
+    N = cfg["N"]
+    B = args.batch or cfg["B"]
+    cap = bvn_capacity(N)
+    warm = max(args.warmup, 3)
+    D_host = make_demand(CFG, B, seed=260526845 + rank)
+    dev = torch.device("cuda", local_rank)
+    d = torch.from_numpy(D_host).to(dev)
+    stream = torch.cuda.current_stream()
+
+    def sched(kcap):
+        return ms.Schedule(perm=torch.empty((B, kcap, N), dtype=torch.uint8, device=dev),
+                           dur=torch.empty((B, kcap), dtype=torch.int32, device=dev),
+                           count=torch.empty(B, dtype=torch.int32, device=dev),
+                           status=torch.empty(B, dtype=torch.int32, device=dev),
+                           work=torch.zeros((B, ms.WORK_FIELDS), dtype=torch.int64, device=dev))
+
+    mw, bv = sched(K_MW), sched(cap)
+    score_mw = torch.empty((5, B), dtype=torch.int64, device=dev)
+    score_bv = torch.empty((5, B), dtype=torch.int64, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    names = ["mw_decompose", "schedule_eval(mw)", "bvn_decompose", "schedule_eval(bvn)"]
+
+    def step(events=None):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)] if events is not None else None
+        if marks: marks[0].record(stream)
+        ms.mw_decompose(d, K_MW, out=mw)
+        if marks: marks[1].record(stream)
+        ms.schedule_eval(d, mw.perm, mw.dur, mw.count, DEFAULT_MODEL, out=score_mw)
+        if marks: marks[2].record(stream)
+        ms.bvn_decompose(d, cap, out=bv)
+        if marks: marks[3].record(stream)
+        ms.schedule_eval(d, bv.perm, bv.dur, bv.count, DEFAULT_MODEL, out=score_bv)
+        if marks:
+            marks[4].record(stream)
+            events.append(marks)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warm):
+        step()
+    barrier()
+
+    # ---- device-resident timing: K steps, L2 flushed (untimed) between steps ----
+    events = []
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        for _ in range(args.steps):
+            flush.fill_(1)
+            step(events)
+        barrier()
+    per_kernel = np.zeros(4)
+    total_ms = 0.0
+    for marks in events:
+        for i in range(4):
+            per_kernel[i] += marks[i].elapsed_time(marks[i + 1])
+        total_ms += marks[0].elapsed_time(marks[4])
+    per_kernel /= args.steps
+
+    # ---- end to end: pinned host demand in, schedules and scores back to pinned host memory ----
+    h_in = torch.from_numpy(D_host).pin_memory()
+    outs = [mw.perm, mw.dur, mw.count, mw.status, bv.perm, bv.dur, bv.count, bv.status, score_mw, score_bv]
+    h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    h2d = h_in.numel() * h_in.element_size()
+    d2h = sum(t.numel() * t.element_size() for t in outs)
+
+    def e2e_step():
+        d.copy_(h_in, non_blocking=True)
+        step()
+        for h, t in zip(h_out, outs):
+            h.copy_(t, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(1, min(args.steps, 3))
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = times.tolist()
+
+    ok = bool((mw.status >= 0).all() and (bv.status == 0).all())
+    work_mw = mw.work.cpu().numpy().astype(np.float64)
+    work_bv = bv.work.cpu().numpy().astype(np.float64)
+
+    if rank == 0:
+        value = world * B * args.steps / (total_ms * 1e-3)
+        ck = clocks.summary()
+        peaks, peak_kind = measured_peaks()
+        sm_mhz = ck["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
+        ops_mw, ops_bvn = algorithmic_ops(work_mw, work_bv, N)
+        dom = int(np.argmax(per_kernel))
+        dom_ops = ops_bvn if dom == 2 else ops_mw
+        alu_peak = ALU_LANES_PER_CLK * sm_mhz * 1e6 / 1e9          # G lane-ops/s at the sampled clock
+        achieved = dom_ops / (per_kernel[dom] * 1e-3) / 1e9
+        k_bv = float(bv.count.double().mean())
+        k_mw = float(mw.count.double().mean())
+        bytes_bvn = B * (4 * N * N + k_bv * (N + 4) + 8)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": workload_name(B), "l2": "flushed between timed steps (256 MiB write, untimed)",
+                       "matchings_per_matrix": {"greedy": k_mw, "bvn": k_bv}, "all_status_ok": ok,
+                       "seed": 260526845},
+            "kernels_ms": {n: float(t) for n, t in zip(names, per_kernel)},
+            "rates": {"greedy_per_s": B / (per_kernel[0] * 1e-3), "bvn_per_s": B / (per_kernel[2] * 1e-3)},
+            "roofline": {"kernel": names[dom], "bound": "alu", "achieved": achieved, "peak": alu_peak,
+                         "unit": "Gop/s", "frac": achieved / alu_peak, "traffic": None,
+                         "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (sampled)",
+                         "hbm_side": {"algorithmic_bytes": bytes_bvn,
+                                      "gbs": bytes_bvn / (per_kernel[2] * 1e-3) / 1e9,
+                                      "peak_gbs": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}"}},
+            "e2e": {"value": world * B * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": 4 * args.steps,
+            "clocks": ck,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            threads = oracle.hardware_threads()
+            sample = min(B, max(threads, 16) * 2)
+            rate = oracle_rate(D_host[:sample], threads, cap)
+            out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                   "sample": f"first {sample} matrices of the same batch, whole path"}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
