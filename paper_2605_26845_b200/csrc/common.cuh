@@ -22,29 +22,31 @@ enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL =
 
 // ---- small helpers on register arrays -------------------------------------------------
 
-template <int W>
-__device__ __forceinline__ unsigned word_of(const unsigned (&m)[W], int idx) {
-  unsigned w = m[0];
-#pragma unroll
-  for (int k = 1; k < W; ++k)
-    if ((idx >> 5) == k) w = m[k];
-  return w;
-}
+// Bit access with a run-time index is written as arithmetic over ALL words (never as
+// "touch word k if idx/32 == k"), so that the compiler cannot turn it into an indexed
+// access that would push the register array into local memory.
 template <int W>
 __device__ __forceinline__ bool test_bit(const unsigned (&m)[W], int idx) {
-  return (word_of<W>(m, idx) >> (idx & 31)) & 1u;
+  const unsigned bit = 1u << (idx & 31);
+  const int wi = idx >> 5;
+  unsigned hit = 0u;
+#pragma unroll
+  for (int k = 0; k < W; ++k) hit |= m[k] & (wi == k ? bit : 0u);
+  return hit != 0u;
 }
 template <int W>
 __device__ __forceinline__ void set_bit(unsigned (&m)[W], int idx) {
+  const unsigned bit = 1u << (idx & 31);
+  const int wi = idx >> 5;
 #pragma unroll
-  for (int k = 0; k < W; ++k)
-    if ((idx >> 5) == k) m[k] |= 1u << (idx & 31);
+  for (int k = 0; k < W; ++k) m[k] |= (wi == k ? bit : 0u);
 }
 template <int W>
 __device__ __forceinline__ void clear_bit(unsigned (&m)[W], int idx) {
+  const unsigned bit = 1u << (idx & 31);
+  const int wi = idx >> 5;
 #pragma unroll
-  for (int k = 0; k < W; ++k)
-    if ((idx >> 5) == k) m[k] &= ~(1u << (idx & 31));
+  for (int k = 0; k < W; ++k) m[k] &= ~(wi == k ? bit : 0u);
 }
 template <int W>
 __device__ __forceinline__ bool any_bit(const unsigned (&m)[W]) {
