@@ -57,6 +57,10 @@ extern "C" {
 
 #define MOESCHED_MAX_N 256
 
+/* Largest entry the greedy decomposition accepts (2^28): its integer duals stay within a
+ * few multiples of the largest entry, which must fit 31 bits. */
+#define MOESCHED_MW_MAX_ENTRY 268435456
+
 /* Number of int64 work counters per matrix written to d_work (see below). */
 #define MOESCHED_WORK_FIELDS 8
 
@@ -85,7 +89,7 @@ typedef struct moesched_model {
  * matched entry (paper Sec. 3.3 / 4.1: the heaviest pair sets the completion
  * time); the matched entries are served whole and set to zero.
  *
- *   d_demand   in   [B][N][N] int32, entries >= 0 and N * max entry <= 2^31-1
+ *   d_demand   in   [B][N][N] int32, 0 <= entry <= MOESCHED_MW_MAX_ENTRY (2^28)
  *   k_max      in   matching budget and output capacity, >= 1
  *   d_perm     out  [B][k_max][N] uint8
  *   d_dur      out  [B][k_max] int32
@@ -95,9 +99,9 @@ typedef struct moesched_model {
  *   d_status   out  [B] int32
  *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64 work counters, may be NULL:
  *                   0 shortest-path column scans, 1 augmentations, 2 rows
- *                   tested for tightness, 3 canonicalisation sweeps that
- *                   searched, 4 search levels, 5 rotation steps, 6 matchings,
- *                   7 unused
+ *                   tried against their best column, 3 canonicalisation
+ *                   sweeps that searched, 4 search levels, 5 rotation steps,
+ *                   6 matchings, 7 unused
  */
 int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                           int32_t* d_dur, int32_t* d_count, int32_t* d_residual,

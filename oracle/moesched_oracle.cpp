@@ -60,6 +60,7 @@ const int ST_BAD_INPUT = -1;
 const int ST_INTERNAL = -2;
 
 const i64 I32_MAX = 2147483647LL;
+const i64 MW_MAX_ENTRY = 1LL << 28;   // input range of the greedy decomposition
 
 // ---------------------------------------------------------------------------
 // Tier 0: enumeration in lexicographic order.
@@ -308,7 +309,7 @@ void mw_one(int tier, int N, const int32_t* D, int k_max, uint8_t* perm, int32_t
     if (D[e] < 0) { *count = 0; *status = ST_BAD_INPUT; return; }
     mx = std::max<i64>(mx, D[e]);
   }
-  if (mx * N > I32_MAX) { *count = 0; *status = ST_BAD_INPUT; return; }
+  if (mx > MW_MAX_ENTRY) { *count = 0; *status = ST_BAD_INPUT; return; }
   std::vector<i64> R(D, D + NN);
   std::vector<int> pi(N);
   int k = 0;

@@ -3,35 +3,43 @@
 // The matrix is balanced by north-west-corner padding, then peeled: the support
 // graph (positive entries) is kept as one row-set bit mask per column in
 // registers; after each subtraction only the rows whose matched entry reached
-// zero are re-matched by an augmenting search, and canonicalise() restores the
-// lexicographically smallest perfect matching, starting at the first row whose
-// column changed (earlier rows provably keep theirs).
+// zero are re-matched by an augmenting search that disturbs as few low rows as
+// possible, and canonicalise() restores the lexicographically smallest perfect
+// matching over the window of rows whose column changed (rows before the first
+// changed row provably keep theirs; rows after the last one were settled earlier
+// and removing edges cannot unsettle them).
 #include "common.cuh"
 
 namespace moesched {
 
 // Augmenting search from free row f over alternating paths of the support graph.
-// Returns false when no augmenting path exists (cannot happen for a balanced matrix).
+// Among all augmenting paths it takes one whose lowest row is as high as possible: the
+// search first uses only rows >= t = f and lowers t to the highest waiting row only when
+// it is stuck, so the rows below the returned path keep their columns. [lo, hi] is widened
+// to cover every row whose column changed. Returns false when no augmenting path exists
+// (cannot happen for a balanced matrix).
 template <int CPL>
 __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], int (&mr)[CPL],
-                                             short* x, int& first_changed, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+                                             short* x, int& lo, int& hi, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
-  unsigned F[W];
+  unsigned F[W], P[W];   // frontier rows; rows met but still below the threshold
 #pragma unroll
-  for (int w = 0; w < W; ++w) F[w] = 0u;
+  for (int w = 0; w < W; ++w) F[w] = P[w] = 0u;
   set_bit<W>(F, f);
+  int t = f;
   unsigned visited = 0u;
   int par[CPL];
 #pragma unroll
   for (int s = 0; s < CPL; ++s) par[s] = -1;
   int jf = -1;
-  for (int it = 0; it < N; ++it) {
-    unsigned nxt[W];
+  for (int it = 0; it < 2 * N + 2; ++it) {
+    unsigned met[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) nxt[w] = 0u;
+    for (int w = 0; w < W; ++w) met[w] = 0u;
     int freeslot = -1;
 #pragma unroll
-    for (int s = CPL - 1; s >= 0; --s) {
+    for (int ss = 0; ss < CPL; ++ss) {
+      const int s = CPL - 1 - ss;
       if (!((visited >> s) & 1u)) {
         unsigned hit[W];
 #pragma unroll
@@ -40,7 +48,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
           visited |= 1u << s;
           par[s] = lowest_bit<W>(hit);
           if (mr[s] < 0) freeslot = s;
-          else set_bit<W>(nxt, mr[s]);
+          else set_bit<W>(met, mr[s]);
         }
       }
     }
@@ -54,10 +62,19 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
     bool grew = false;
 #pragma unroll
     for (int w = 0; w < W; ++w) {
-      F[w] = __reduce_or_sync(FULL, nxt[w]);
+      const unsigned m = __reduce_or_sync(FULL, met[w]);
+      const unsigned ge = ge_word(t, w);
+      F[w] = m & ge;
+      P[w] |= m & ~ge;
       grew |= F[w] != 0u;
     }
-    if (!grew) return false;
+    if (!grew) {
+      const int r = highest_bit<W>(P);   // admit the highest waiting row, and only that one
+      if (r < 0) return false;
+      t = r;
+      clear_bit<W>(P, r);
+      set_bit<W>(F, r);
+    }
   }
   if (jf < 0) return false;
   int j = jf;
@@ -69,7 +86,8 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
     if (lane == L) put<CPL>(mr, sl, i);
     if (lane == 0) x[i] = (short)j;
     __syncwarp();
-    first_changed = min(first_changed, i);
+    lo = min(lo, i);
+    hi = max(hi, i);
     work[WK_AUG]++;
     if (i == f) return true;
     j = jprev;
@@ -192,7 +210,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 
     uint8_t* pout = perm + (size_t)b * k_max * N;
     int32_t* cout_ = coef + (size_t)b * k_max;
-    int first_changed = 0;
+    int lo_changed = 0, hi_changed = N - 1;   // window of rows whose column may not be final
     unsigned freerows[W];   // uniform: rows without a column
 #pragma unroll
     for (int w = 0; w < W; ++w) {
@@ -206,13 +224,15 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       for (int it = 0; it < N; ++it) {
         const int f = lowest_bit<W>(freerows);
         if (f < 0) break;
-        first_changed = min(first_changed, f);
-        if (!augment_from<CPL>(N, lane, f, C, mr, x, first_changed, work)) { okm = false; break; }
+        if (!augment_from<CPL>(N, lane, f, C, mr, x, lo_changed, hi_changed, work)) { okm = false; break; }
         clear_bit<W>(freerows, f);
       }
       if (!okm || any_bit<W>(freerows)) { st_code = MOESCHED_ST_INTERNAL; break; }
-      work[WK_SKIP] += first_changed;
-      if (!canonicalise<CPL>(N, lane, first_changed, C, mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      work[WK_SKIP] += lo_changed;
+      if (!canonicalise<CPL>(N, lane, lo_changed, hi_changed, C, mr, x, hist, work)) {
+        st_code = MOESCHED_ST_INTERNAL;
+        break;
+      }
 
       // coefficient = smallest matched entry; subtract it along the matching
       int val[CPL], cmin = INF32;
@@ -223,7 +243,8 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
         if (c < N) { val[s] = A.row(mr[s])[c]; cmin = min(cmin, val[s]); }
       }
       cmin = __reduce_min_sync(FULL, cmin);
-      first_changed = N;
+      lo_changed = N;
+      hi_changed = -1;
       unsigned gone[W];
 #pragma unroll
       for (int w = 0; w < W; ++w) gone[w] = 0u;

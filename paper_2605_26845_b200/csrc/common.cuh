@@ -64,6 +64,20 @@ __device__ __forceinline__ int lowest_bit(const unsigned (&m)[W]) {
     if (m[k]) r = k * 32 + __ffs(m[k]) - 1;
   return r;
 }
+// highest set bit of a mask, or -1
+template <int W>
+__device__ __forceinline__ int highest_bit(const unsigned (&m)[W]) {
+  int r = -1;
+#pragma unroll
+  for (int k = 0; k < W; ++k)
+    if (m[k]) r = k * 32 + 31 - __clz(m[k]);
+  return r;
+}
+// word k of the set {t, t+1, ...}
+__device__ __forceinline__ unsigned ge_word(int t, int k) {
+  const int lo = k * 32;
+  return t <= lo ? 0xffffffffu : (t >= lo + 32 ? 0u : (0xffffffffu << (t - lo)));
+}
 template <int C, typename T>
 __device__ __forceinline__ T pick(const T (&a)[C], int s) {
   T v = a[0];
@@ -274,16 +288,22 @@ __device__ __forceinline__ void cluster_epilogue() {
 // State: C[s] = set of rows adjacent to the lane's column s in the graph (tight
 // edges for the greedy step, positive entries for Birkhoff), mr[s] = row matched
 // to that column, x[r] = column matched to row r (shared memory, one entry per
-// row). On entry (mr, x) is some perfect matching of the graph that already
-// agrees with the answer on rows < start. For each row i >= start in order the
-// routine finds the lowest column that row i can take in a perfect matching that
-// keeps rows < i fixed: an edge (i, j) outside the matching is usable iff row
-// mr[j] reaches row i along alternating steps r -> r' (r adjacent to the column
-// of r') among the rows not yet fixed; the matching is then rotated along that
-// cycle. hist holds one row set per search level to retrace the cycle.
+// row). On entry (mr, x) is some perfect matching of the graph. For each row i
+// in order the routine finds the lowest column that row i can take in a perfect
+// matching that keeps rows < i fixed: an edge (i, j) outside the matching is
+// usable iff row mr[j] reaches row i along alternating steps r -> r' (r adjacent
+// to the column of r') among the rows not yet fixed; the matching is then rotated
+// along that cycle. hist holds one row set per search level to retrace the cycle.
+//
+// Only the window [start, last] of rows is visited. The caller guarantees that the
+// matching already equals the answer on rows < start, and that every row > last
+// was settled by an earlier call, with no row >= it re-matched and no edge added
+// since: its search could only find less now, so its column stands. A rotation at
+// row i moves rows above i and widens the window accordingly.
 template <int CPL>
-__device__ __forceinline__ bool canonicalise(int N, int lane, int start, const unsigned (&C)[CPL][CPL],
-                                             int (&mr)[CPL], short* x, unsigned* hist,
+__device__ __forceinline__ bool canonicalise(int N, int lane, int start, int last,
+                                             const unsigned (&C)[CPL][CPL], int (&mr)[CPL], short* x,
+                                             unsigned* hist,
                                              unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   bool ok_all = true;
@@ -296,7 +316,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, const u
     if (N < hi) m &= N <= lo ? 0u : (0xffffffffu >> (hi - N));
     alive[w] = m;
   }
-  for (int i = start; i < N; ++i) {
+  for (int i = start; i <= last && i < N; ++i) {
     const int xi = x[i];
     // columns below the current one that row i is adjacent to and whose row is still free to move
     bool cand = false;
@@ -378,6 +398,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, const u
         const int nxt = __shfl_sync(FULL, pick<CPL>(mr, s2), L2);
         if (lane == L2) put<CPL>(mr, s2, cur);
         if (lane == 0) x[cur] = (short)(L2 * CPL + s2);
+        last = max(last, cur);
         cur = nxt;
         --lvl;
         work[WK_ROT]++;

@@ -2,9 +2,9 @@
 //
 // Each greedy step solves one assignment problem on the residual matrix R by
 // shortest augmenting paths on cost = -R (a Jonker-Volgenant style search that
-// keeps only the column duals v and settles one column per scan), derives the
-// row duals, marks the tight edges and hands that graph to canonicalise(), which
-// returns the lexicographically smallest optimal permutation. The matched
+// keeps only the column duals v, warm-started from the previous step), derives
+// the row duals, marks the tight edges and hands that graph to canonicalise(),
+// which returns the lexicographically smallest optimal permutation. The matched
 // entries are then served whole; the largest one is the matching's duration.
 #include "common.cuh"
 
@@ -16,16 +16,60 @@ struct MwState {
   int mr[CPL];    // row assigned to the lane's column, -1 if free
 };
 
-// One assignment problem from scratch. Returns false if an iteration limit was hit.
+// One assignment problem. The column duals v carry over from the previous greedy step
+// (weights only decreased, so they are still feasible); they are shifted so that the largest
+// is zero, which keeps every intermediate value within a few multiples of the largest entry.
+// Each row first tries the column that minimises cost - v (lowest column on ties) and keeps
+// it if that column is still free: such a row is matched along a tight edge. The rows left
+// over are added one by one by a shortest-augmenting-path search that settles one column
+// per scan and updates only the column duals. Returns false if an iteration limit was hit.
 template <int CPL>
 __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int lane, bool lane_in,
                                                  MwState<CPL>& st, short* x, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = CPL;
   bool ok = true;
+  {
+    int vmax = -INF32;
 #pragma unroll
-  for (int s = 0; s < CPL; ++s) { st.v[s] = 0; st.mr[s] = -1; }
+    for (int s = 0; s < CPL; ++s)
+      if (lane * CPL + s < N) vmax = max(vmax, st.v[s]);
+    vmax = __reduce_max_sync(FULL, vmax);
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) { st.v[s] -= vmax; st.mr[s] = -1; }
+  }
   for (int r = lane; r < N; r += 32) x[r] = -1;
+  unsigned freerows[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) freerows[w] = 0u;
   __syncwarp();
-  for (int f = 0; f < N; ++f) {
+  for (int r = 0; r < N; ++r) {
+    RowVec<CPL> rv;
+    if (lane_in) rv = load_cols<CPL>(R.row(r), lane);
+    int lmin = INF32, lslot = 0;
+#pragma unroll
+    for (int ss = 0; ss < CPL; ++ss) {
+      const int s = CPL - 1 - ss;
+      const int d = (lane * CPL + s < N) ? -rv.v[s] - st.v[s] : INF32;
+      if (d <= lmin) { lmin = d; lslot = s; }
+    }
+    const int u = __reduce_min_sync(FULL, lmin);
+    const unsigned ball = __ballot_sync(FULL, lmin == u);
+    const int L = __ffs(ball) - 1;
+    const int sl = __shfl_sync(FULL, lslot, L);
+    const int owner = __shfl_sync(FULL, pick<CPL>(st.mr, sl), L);
+    if (owner < 0) {
+      if (lane == L) put<CPL>(st.mr, sl, r);
+      if (lane == 0) x[r] = (short)(L * CPL + sl);
+    } else {
+      set_bit<W>(freerows, r);
+    }
+    work[WK_TIGHT]++;
+  }
+  __syncwarp();
+  for (int outer = 0; outer < N; ++outer) {
+    const int f = lowest_bit<W>(freerows);
+    if (f < 0) break;
+    clear_bit<W>(freerows, f);
     int dist[CPL], pred[CPL];
     unsigned scanned = 0u;     // bit s: the lane's column s is settled
     {
@@ -43,7 +87,8 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
     for (int it = 0; it < N; ++it) {
       int lmin = INF32, lslot = 0;
 #pragma unroll
-      for (int s = CPL - 1; s >= 0; --s) {
+      for (int ss = 0; ss < CPL; ++ss) {
+        const int s = CPL - 1 - ss;
         int d = ((scanned >> s) & 1u) ? INF32 : dist[s];
         if (d <= lmin) { lmin = d; lslot = s; }
       }
@@ -87,6 +132,7 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
     }
     work[WK_AUG]++;
   }
+  if (any_bit<W>(freerows)) ok = false;
   return ok;
 }
 
@@ -133,12 +179,14 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
     neg = __any_sync(FULL, neg);
     mx = __reduce_max_sync(FULL, mx);
     nnz = __reduce_add_sync(FULL, cnt);
-    if (neg || (long long)mx * N > 2147483647LL) st_code = MOESCHED_ST_BAD_INPUT;
+    if (neg || mx > MOESCHED_MW_MAX_ENTRY) st_code = MOESCHED_ST_BAD_INPUT;
     if (!loaded) st_code = MOESCHED_ST_INTERNAL;
   }
 
   if (st_code == MOESCHED_ST_OK) {
     MwState<CPL> st;
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) { st.v[s] = 0; st.mr[s] = -1; }
     uint8_t* pout = perm + (size_t)b * k_max * N;
     int32_t* dout = dur + (size_t)b * k_max;
     while (k < k_max && nnz > 0) {
@@ -168,8 +216,7 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
             if (red[s] == u && lane * CPL + s < N) C[s][w] |= 1u << q;
         }
       }
-      work[WK_TIGHT] += N;
-      if (!canonicalise<CPL>(N, lane, 0, C, st.mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      if (!canonicalise<CPL>(N, lane, 0, N - 1, C, st.mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
       // serve: the heaviest matched pair sets the duration; matched entries are sent whole
       int dmax = 0, served = 0;
 #pragma unroll

@@ -86,7 +86,7 @@ def test_closed_form_cases(N):
 def test_bad_inputs_and_budget():
     D = make_demand(1, 6)
     D[1, 2, 3] = -1
-    D[4, 0, 0] = 2**31 - 1          # N * max entry and the row sum overflow 31 bits
+    D[4, 0, 0] = 2**31 - 1          # entry above 2^28 (greedy) and row sum beyond 31 bits (BvN)
     check_all(D, 8, 50)
     check_all(D, 1, 1)
     check_all(D, 3, 7)

@@ -197,7 +197,7 @@ def test_bad_input_status():
     for out in (g, v):
         assert list(out["status"]) == [0, -1, 0] and out["count"][1] == 0
     big = np.zeros((1, 8, 8), np.int32)
-    big[0, 0, 0] = 2**31 - 1                                      # N * max entry must fit 31 bits (greedy)
+    big[0, 0, 0] = 2**31 - 1                                      # entries above 2^28 are out of range for the greedy path
     assert oracle.mw_decompose(big, 8)["status"][0] == -1
     assert oracle.bvn_decompose(big, 50)["status"][0] == 0
     big[0, 0, 1] = 1                                              # row sum overflows 31 bits (BvN)
