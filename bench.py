@@ -201,6 +201,7 @@ def main():
     score_mw = torch.empty((5, B), dtype=torch.int64, device=dev)
     score_bv = torch.empty((5, B), dtype=torch.int64, device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    scratch = torch.empty(ms.bvn_scratch_bytes(B, N), dtype=torch.uint8, device=dev)
 
     names = ["mw_decompose", "schedule_eval(mw)", "bvn_decompose", "schedule_eval(bvn)"]
 
@@ -211,7 +212,7 @@ def main():
         if marks: marks[1].record(stream)
         ms.schedule_eval(d, mw.perm, mw.dur, mw.count, DEFAULT_MODEL, out=score_mw)
         if marks: marks[2].record(stream)
-        ms.bvn_decompose(d, cap, out=bv)
+        ms.bvn_decompose(d, cap, out=bv, scratch=scratch)
         if marks: marks[3].record(stream)
         ms.schedule_eval(d, bv.perm, bv.dur, bv.count, DEFAULT_MODEL, out=score_bv)
         if marks:

@@ -128,6 +128,14 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
  *   d_coef     out  [B][k_max] int32 coefficients c_k (tokens per pair)
  *   d_count    out  [B] int32
  *   d_aug      out  [B][N][N] int32 the balanced matrix A; may be NULL
+ *   d_scratch  tmp  moesched_bvn_scratch_bytes(B, N) bytes of device memory, 32-byte
+ *                   aligned, or NULL. With scratch the working copy of every matrix
+ *                   lives there (it stays in L2) and shared memory is left for
+ *                   bookkeeping, so several times more matrices are in flight per SM:
+ *                   the fast path. Without it the matrix is held in shared memory
+ *                   (a 2-CTA cluster for N > 232). Results are identical. Contents
+ *                   are undefined afterwards; calls that overlap in time need
+ *                   separate scratch.
  *   d_status   out  [B] int32
  *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64, may be NULL: 0 augmenting
  *                   search levels, 1 augmenting-path steps, 2 matchings
@@ -136,8 +144,12 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
  *                   skipped as unchanged prefix
  */
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
-                           int32_t* d_coef, int32_t* d_count, int32_t* d_aug,
+                           int32_t* d_coef, int32_t* d_count, int32_t* d_aug, int32_t* d_scratch,
                            int32_t* d_status, int64_t* d_work, void* stream);
+
+/* Bytes of scratch that moesched_bvn_decompose can use for B matrices of size N
+ * (B * N * roundup(N, 8) * 4); 0 for sizes out of range. */
+size_t moesched_bvn_scratch_bytes(int B, int N);
 
 /*
  * Score a schedule (paper Sec. 4.1: a matching completes after its largest

@@ -49,6 +49,7 @@ def load_library():
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval",
                      "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
+        lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         _lib = lib
     return _lib
 
@@ -89,37 +90,71 @@ class Schedule:
     work: torch.Tensor | None = None
 
 
-def _decompose(fn_name, demand, k_max, want_extra, want_work, out):
-    lib = load_library()
+def _new_schedule(demand, k_max, want_extra, want_work):
+    B, N, _ = demand.shape
+    dev = demand.device
+    return Schedule(perm=torch.empty((B, k_max, N), dtype=torch.uint8, device=dev),
+                    dur=torch.empty((B, k_max), dtype=torch.int32, device=dev),
+                    count=torch.empty(B, dtype=torch.int32, device=dev),
+                    status=torch.empty(B, dtype=torch.int32, device=dev),
+                    extra=torch.empty_like(demand) if want_extra else None,
+                    work=torch.empty((B, WORK_FIELDS), dtype=torch.int64, device=dev) if want_work else None)
+
+
+def _check_demand(demand):
     demand = _dev(demand, torch.int32, "demand")
     if demand.dim() != 3 or demand.shape[1] != demand.shape[2]:
         raise MoeschedError("demand must have shape [B, N, N]")
-    B, N, _ = demand.shape
-    dev = demand.device
-    if out is None:
-        out = Schedule(perm=torch.empty((B, k_max, N), dtype=torch.uint8, device=dev),
-                       dur=torch.empty((B, k_max), dtype=torch.int32, device=dev),
-                       count=torch.empty(B, dtype=torch.int32, device=dev),
-                       status=torch.empty(B, dtype=torch.int32, device=dev),
-                       extra=torch.empty_like(demand) if want_extra else None,
-                       work=torch.empty((B, WORK_FIELDS), dtype=torch.int64, device=dev) if want_work else None)
-    with torch.cuda.device(dev):
-        rc = getattr(lib, fn_name)(B, N, _ptr(demand), int(k_max), _ptr(out.perm), _ptr(out.dur), _ptr(out.count),
-                                   _ptr(out.extra), _ptr(out.status), _ptr(out.work), _stream(dev))
-    _check(rc, fn_name)
-    return out
+    return demand
 
 
 def mw_decompose(demand, k_max, want_residual=False, want_work=False, out=None) -> Schedule:
     """Greedy max-weight decomposition of every matrix of `demand` [B, N, N] int32 (CUDA)."""
-    return _decompose("moesched_mw_decompose", demand, k_max, want_residual, want_work, out)
+    lib = load_library()
+    demand = _check_demand(demand)
+    B, N, _ = demand.shape
+    dev = demand.device
+    if out is None:
+        out = _new_schedule(demand, int(k_max), want_residual, want_work)
+    with torch.cuda.device(dev):
+        rc = lib.moesched_mw_decompose(B, N, _ptr(demand), int(k_max), _ptr(out.perm), _ptr(out.dur),
+                                       _ptr(out.count), _ptr(out.extra), _ptr(out.status), _ptr(out.work),
+                                       _stream(dev))
+    _check(rc, "moesched_mw_decompose")
+    return out
 
 
-def bvn_decompose(demand, k_max=None, want_aug=False, want_work=False, out=None) -> Schedule:
-    """Birkhoff-von Neumann decomposition; k_max defaults to N^2 - 2N + 2 (always enough)."""
+def bvn_scratch_bytes(B, N) -> int:
+    return int(load_library().moesched_bvn_scratch_bytes(int(B), int(N)))
+
+
+def bvn_decompose(demand, k_max=None, want_aug=False, want_work=False, out=None, scratch=True) -> Schedule:
+    """Birkhoff-von Neumann decomposition; k_max defaults to N^2 - 2N + 2 (always enough).
+
+    scratch: True allocates the working buffer of the fast path, a uint8 CUDA tensor of at least
+    bvn_scratch_bytes(B, N) bytes is used as given, False / None selects the shared-memory path."""
+    lib = load_library()
+    demand = _check_demand(demand)
+    B, N, _ = demand.shape
+    dev = demand.device
     if k_max is None:
-        k_max = bvn_capacity(demand.shape[1])
-    return _decompose("moesched_bvn_decompose", demand, k_max, want_aug, want_work, out)
+        k_max = bvn_capacity(N)
+    if out is None:
+        out = _new_schedule(demand, int(k_max), want_aug, want_work)
+    if scratch is True:
+        scratch = torch.empty(max(1, bvn_scratch_bytes(B, N)), dtype=torch.uint8, device=dev)
+    elif scratch is False:
+        scratch = None
+    if scratch is not None:
+        _dev(scratch, torch.uint8, "scratch")
+        if scratch.numel() < bvn_scratch_bytes(B, N):
+            raise MoeschedError("scratch is smaller than bvn_scratch_bytes(B, N)")
+    with torch.cuda.device(dev):
+        rc = lib.moesched_bvn_decompose(B, N, _ptr(demand), int(k_max), _ptr(out.perm), _ptr(out.dur),
+                                        _ptr(out.count), _ptr(out.extra), _ptr(scratch), _ptr(out.status),
+                                        _ptr(out.work), _stream(dev))
+    _check(rc, "moesched_bvn_decompose")
+    return out
 
 
 SCORE_FIELDS = ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",

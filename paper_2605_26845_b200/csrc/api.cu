@@ -53,15 +53,21 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }
 
+size_t moesched_bvn_scratch_bytes(int B, int N) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N) return 0;
+  return (size_t)B * N * bvn_scratch_stride(N) * sizeof(int32_t);
+}
+
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm, int32_t* d_coef,
-                           int32_t* d_count, int32_t* d_aug, int32_t* d_status, int64_t* d_work, void* stream) {
+                           int32_t* d_count, int32_t* d_aug, int32_t* d_scratch, int32_t* d_status,
+                           int64_t* d_work, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
   if (!d_demand || !d_perm || !d_coef || !d_count || !d_status) return MOESCHED_EINVAL;
   if (!aligned4(d_demand) || !aligned4(d_coef) || !aligned4(d_count) || !aligned4(d_status) || !aligned4(d_aug) ||
-      !aligned8(d_work))
+      !aligned8(d_work) || (reinterpret_cast<uintptr_t>(d_scratch) & 31) != 0)
     return MOESCHED_EINVAL;
   if (B == 0) return MOESCHED_OK;
-  cudaError_t e = run_bvn(B, N, d_demand, k_max, d_perm, d_coef, d_count, d_aug, d_status,
+  cudaError_t e = run_bvn(B, N, d_demand, k_max, d_perm, d_coef, d_count, d_aug, d_scratch, d_status,
                           reinterpret_cast<long long*>(d_work), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }

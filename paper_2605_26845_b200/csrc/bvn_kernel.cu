@@ -96,14 +96,20 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   return false;
 }
 
-template <int CPL, bool CLUSTER>
+// MODE 0: matrix in this CTA's shared memory; 1: split over a 2-CTA cluster; 2: working copy
+// in global memory (scratch), which leaves room for many more warps per SM.
+template <int CPL, int MODE>
 __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                   uint8_t* __restrict__ perm, int32_t* __restrict__ coef,
                                                   int32_t* __restrict__ count, int32_t* __restrict__ aug,
-                                                  int32_t* __restrict__ status, long long* __restrict__ work_out) {
+                                                  int32_t* scratch, int32_t* __restrict__ status,
+                                                  long long* __restrict__ work_out) {
   constexpr int W = CPL;
+  constexpr bool CLUSTER = MODE == 1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+  WarpCtx cx;
+  if constexpr (MODE == 2) cx = warp_prologue_global<CPL>(B, N, S, demand, scratch, smem_raw);
+  else cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
   if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
   const int lane = cx.lane, b = cx.b;
   const MatView A = cx.M;
@@ -296,17 +302,30 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 // ---- host side ---------------------------------------------------------------------------
 
 cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
-                    int32_t* aug, int32_t* status, long long* work, cudaStream_t stream) {
-  const Geometry ge = plan_geometry(N);
-#define MOESCHED_GO(C, CL)                                                                                    \
-  return launch_warp_kernel(bvn_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, count, \
-                            aug, status, work)
-  if (ge.cluster) MOESCHED_GO(8, true);
+                    int32_t* aug, int32_t* scratch, int32_t* status, long long* work, cudaStream_t stream) {
+  Geometry ge = plan_geometry(N);
+#define MOESCHED_GO(C, M)                                                                                    \
+  return launch_warp_kernel(bvn_kernel<C, M>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, count, \
+                            aug, scratch, status, work)
+  if (scratch != nullptr) {
+    // working copy in global memory: four matrices per CTA, shared memory only for hist and x
+    ge.cluster = false;
+    ge.S = bvn_scratch_stride(N);
+    ge.wpb = 4;
+    ge.smem = warp_smem_bytes_global(N, ge.cpl) * ge.wpb;
+    switch (ge.cpl) {
+      case 1: MOESCHED_GO(1, 2);
+      case 2: MOESCHED_GO(2, 2);
+      case 4: MOESCHED_GO(4, 2);
+      default: MOESCHED_GO(8, 2);
+    }
+  }
+  if (ge.cluster) MOESCHED_GO(8, 1);
   switch (ge.cpl) {
-    case 1: MOESCHED_GO(1, false);
-    case 2: MOESCHED_GO(2, false);
-    case 4: MOESCHED_GO(4, false);
-    default: MOESCHED_GO(8, false);
+    case 1: MOESCHED_GO(1, 0);
+    case 2: MOESCHED_GO(2, 0);
+    case 4: MOESCHED_GO(4, 0);
+    default: MOESCHED_GO(8, 0);
   }
 #undef MOESCHED_GO
 }

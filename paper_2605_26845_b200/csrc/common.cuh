@@ -277,6 +277,39 @@ __device__ __forceinline__ WarpCtx warp_prologue(int B, int N, int S, const int3
   return cx;
 }
 
+// Variant with the working copy of the matrix in caller-provided global memory (row stride
+// S ints, one N x S slab per matrix): shared memory then holds only hist and x, so many more
+// warps fit on an SM. Suits kernels that touch the matrix a few times per matching.
+__host__ __device__ inline size_t warp_smem_bytes_global(int N, int W) {
+  return align16((size_t)(N + 1) * W * 4) + align16((size_t)N * 2);
+}
+
+template <int CPL>
+__device__ __forceinline__ WarpCtx warp_prologue_global(int B, int N, int S, const int32_t* demand,
+                                                        int32_t* scratch, unsigned char* smem_raw) {
+  WarpCtx cx;
+  cx.lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int wpb = blockDim.x >> 5;
+  unsigned char* base = smem_raw + (size_t)warp * warp_smem_bytes_global(N, CPL);
+  cx.hist = reinterpret_cast<unsigned*>(base);
+  cx.x = reinterpret_cast<short*>(base + align16((size_t)(N + 1) * CPL * 4));
+  cx.b = blockIdx.x * wpb + warp;
+  cx.worker = cx.b < B;
+  cx.loaded = true;
+  cx.M.S = S;
+  cx.M.split = N;
+  cx.M.near_ = cx.M.far_ = nullptr;
+  if (!cx.worker) return cx;
+  int* mat = scratch + (size_t)cx.b * N * S;
+  cx.M.near_ = cx.M.far_ = mat;
+  const int32_t* src = demand + (size_t)cx.b * N * N;
+  for (int r = 0; r < N; ++r)
+    for (int c = cx.lane; c < S; c += 32) mat[(size_t)r * S + c] = c < N ? src[(size_t)r * N + c] : 0;
+  __syncwarp();
+  return cx;
+}
+
 // Every warp of a cluster launch passes here exactly once before it returns.
 template <bool CLUSTER>
 __device__ __forceinline__ void cluster_epilogue() {
@@ -300,40 +333,71 @@ __device__ __forceinline__ void cluster_epilogue() {
 // was settled by an earlier call, with no row >= it re-matched and no edge added
 // since: its search could only find less now, so its column stands. A rotation at
 // row i moves rows above i and widens the window accordingly.
+// Rows i that have, below their own column, a column they are adjacent to whose row lies
+// above i: only those can move to a lower column. Uniform result. With gt(c) = rows matched
+// to a column > c (a suffix OR over the lanes), row i qualifies through column c iff
+// i is adjacent to c, i < mr[c] and i is in gt(c).
+template <int CPL>
+__device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL][CPL], const int (&mr)[CPL],
+                                               unsigned (&cand)[CPL]) {
+  constexpr int W = CPL;
+  unsigned own[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) own[w] = 0u;
+#pragma unroll
+  for (int s = 0; s < CPL; ++s)
+    if (mr[s] >= 0) set_bit<W>(own, mr[s]);
+  unsigned above[W];   // rows matched to the columns of higher lanes
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    unsigned v = own[w];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned t = __shfl_down_sync(FULL, v, o);
+      if (lane + o < 32) v |= t;
+    }
+    const unsigned t = __shfl_down_sync(FULL, v, 1);
+    above[w] = lane < 31 ? t : 0u;
+  }
+  unsigned acc[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+  for (int ss = 0; ss < CPL; ++ss) {
+    const int s = CPL - 1 - ss;   // from the lane's highest column down, growing gt as we go
+    if (mr[s] >= 0) {
+#pragma unroll
+      for (int w = 0; w < W; ++w) acc[w] |= C[s][w] & above[w] & ~ge_word(mr[s], w);
+      set_bit<W>(above, mr[s]);
+    }
+  }
+#pragma unroll
+  for (int w = 0; w < W; ++w) cand[w] = __reduce_or_sync(FULL, acc[w]);
+}
+
 template <int CPL>
 __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int last,
                                              const unsigned (&C)[CPL][CPL], int (&mr)[CPL], short* x,
-                                             unsigned* hist,
-                                             unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+                                             unsigned* hist, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   bool ok_all = true;
-  unsigned alive[W];
+  unsigned cand[W];
+  candidate_rows<CPL>(lane, C, mr, cand);
+  int from = start;
+  for (int guard = 0; guard < N; ++guard) {
+    // next row of the window that could move
+    unsigned todo[W];
 #pragma unroll
-  for (int w = 0; w < W; ++w) {
-    int lo = w * 32, hi = lo + 32;
-    unsigned m = 0xffffffffu;
-    if (start > lo) m = start >= hi ? 0u : (0xffffffffu << (start - lo));
-    if (N < hi) m &= N <= lo ? 0u : (0xffffffffu >> (hi - N));
-    alive[w] = m;
-  }
-  for (int i = start; i <= last && i < N; ++i) {
+    for (int w = 0; w < W; ++w) todo[w] = cand[w] & ge_word(from, w);
+    const int i = lowest_bit<W>(todo);
+    if (i < 0 || i > last) break;
+    from = i + 1;
     const int xi = x[i];
-    // columns below the current one that row i is adjacent to and whose row is still free to move
-    bool cand = false;
-#pragma unroll
-    for (int s = 0; s < CPL; ++s) {
-      int c = lane * CPL + s;
-      cand |= (c < xi) && test_bit<W>(C[s], i) && (mr[s] > i);
-    }
-    if (__ballot_sync(FULL, cand) == 0u) {
-      clear_bit<W>(alive, i);
-      continue;
-    }
     work[WK_SWEEP]++;
-    // backward search from row i
-    unsigned anc[W], F[W];
+    // backward search from row i among the rows >= i
+    unsigned anc[W], F[W], alive[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) anc[w] = F[w] = 0u;
+    for (int w = 0; w < W; ++w) { anc[w] = F[w] = 0u; alive[w] = ge_word(i, w); }
     set_bit<W>(anc, i);
     set_bit<W>(F, i);
     int level = 0;
@@ -363,13 +427,15 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       if (lane < W) hist[level * W + lane] = pick<W>(F, lane);
     }
     __syncwarp();
-    // lowest column row i may take
+    // lowest column row i may take (its own column always qualifies)
     int myslot = -1;
 #pragma unroll
-    for (int s = CPL - 1; s >= 0; --s)
+    for (int ss = 0; ss < CPL; ++ss) {
+      const int s = CPL - 1 - ss;
       if (mr[s] >= 0 && test_bit<W>(C[s], i) && test_bit<W>(anc, mr[s])) myslot = s;
+    }
     unsigned ball = __ballot_sync(FULL, myslot >= 0);
-    if (ball == 0u) { ok_all = false; clear_bit<W>(alive, i); continue; }   // cannot happen: column xi qualifies
+    if (ball == 0u) { ok_all = false; continue; }
     const int L = __ffs(ball) - 1;
     const int sl = __shfl_sync(FULL, myslot, L);
     const int jstar = L * CPL + sl;
@@ -389,8 +455,10 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         for (int w = 0; w < W; ++w) Hm[w] = hist[(lvl - 1) * W + w];
         int ms = -1;
 #pragma unroll
-        for (int s = CPL - 1; s >= 0; --s)
+        for (int ss = 0; ss < CPL; ++ss) {
+          const int s = CPL - 1 - ss;
           if (mr[s] >= 0 && test_bit<W>(Hm, mr[s]) && test_bit<W>(C[s], cur)) ms = s;
+        }
         unsigned b2 = __ballot_sync(FULL, ms >= 0);
         if (b2 == 0u) { ok_all = false; break; }
         const int L2 = __ffs(b2) - 1;
@@ -406,8 +474,8 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       if (lane == L) put<CPL>(mr, sl, i);
       if (lane == 0) x[i] = (short)jstar;
       __syncwarp();
+      candidate_rows<CPL>(lane, C, mr, cand);
     }
-    clear_bit<W>(alive, i);
   }
   return ok_all;
 }
@@ -425,7 +493,9 @@ Geometry plan_geometry(int N);
 cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
                    int32_t* residual, int32_t* status, long long* work, cudaStream_t stream);
 cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
-                    int32_t* aug, int32_t* status, long long* work, cudaStream_t stream);
+                    int32_t* aug, int32_t* scratch, int32_t* status, long long* work, cudaStream_t stream);
+// row stride (ints) of the global working copy used by the Birkhoff kernel
+inline int bvn_scratch_stride(int N) { return (N + 7) / 8 * 8; }
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,

@@ -41,7 +41,10 @@ def test_argument_validation_needs_no_gpu(lib):
     null = ctypes.c_void_p(None)
     assert lib.moesched_mw_decompose(1, 0, null, 1, null, null, null, null, null, null, null) == -1
     assert lib.moesched_mw_decompose(1, 8, null, 1, null, null, null, null, null, null, null) == -1
-    assert lib.moesched_bvn_decompose(1, 257, null, 1, null, null, null, null, null, null, null) == -1
+    assert lib.moesched_bvn_decompose(1, 257, null, 1, null, null, null, null, null, null, null, null) == -1
+    assert lib.moesched_bvn_scratch_bytes(2, 64) == 2 * 64 * 64 * 4
+    assert lib.moesched_bvn_scratch_bytes(1, 17) == 17 * 24 * 4
+    assert lib.moesched_bvn_scratch_bytes(1, 300) == 0
     assert lib.moesched_schedule_eval(1, 8, null, 1, null, null, null, null, null, null, null, null, null,
                                       null, null) == -1
     assert lib.moesched_strerror(0) == b"ok"

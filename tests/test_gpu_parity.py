@@ -37,11 +37,12 @@ def check_all(D, k_mw, k_bvn, model=DEFAULT_MODEL, threads=8):
     assert_schedule_equal(g, rg, "dur")
     ok = rg["status"] >= 0
     assert (g.extra.cpu().numpy()[ok] == rg["residual"][ok]).all()
-    v = ms.bvn_decompose(d, k_bvn, want_aug=True)
     rv = oracle.bvn_decompose(D, k_bvn, threads=threads)
-    assert_schedule_equal(v, rv, "coef")
     ok = rv["status"] >= 0
-    assert (v.extra.cpu().numpy()[ok] == rv["aug"][ok]).all()
+    for scratch in (True, False):       # global working copy / shared-memory (cluster) path
+        v = ms.bvn_decompose(d, k_bvn, want_aug=True, scratch=scratch)
+        assert_schedule_equal(v, rv, "coef")
+        assert (v.extra.cpu().numpy()[ok] == rv["aug"][ok]).all()
     for sched, ref, key in ((g, rg, "dur"), (v, rv, "coef")):
         good = dev(ref["status"] >= 0)
         count = torch.where(good, sched.count, torch.zeros_like(sched.count))
