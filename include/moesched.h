@@ -49,6 +49,7 @@ extern "C" {
 #define MOESCHED_OK 0
 #define MOESCHED_EINVAL (-1)
 #define MOESCHED_ECUDA (-2)
+#define MOESCHED_ETOOBIG (-3)
 
 #define MOESCHED_ST_OK 0
 #define MOESCHED_ST_TRUNCATED 1
@@ -186,6 +187,36 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride,
                            int64_t* d_makespan_serial_ns, int64_t* d_compute_idle_ns,
                            int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
                            int32_t* d_status, void* stream);
+
+/*
+ * Birkhoff-von Neumann decomposition for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of moesched_bvn_decompose,
+ * same arguments, same results, minus d_scratch.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework that
+ * owns the whole memory pool and hands out no raw allocations, in a plug-in or callback
+ * that must not touch the allocator, or in a latency-critical loop where an allocation
+ * (which may synchronise the device) is not acceptable. Such a caller passes inputs and
+ * outputs it already has and still gets the fast path, because the working copy of the
+ * matrices lives in an array built into the library: MOESCHED_STATIC_SCRATCH_BYTES of
+ * device memory that every GPU using the library gives up from load until process exit.
+ *
+ * Limit: B * N * roundup(N, 8) * 4 bytes must not exceed MOESCHED_STATIC_SCRATCH_BYTES
+ * (e.g. B <= 1024 at N = 64, B <= 64 at N = 256); larger batches return MOESCHED_ETOOBIG
+ * and enqueue nothing -- split the batch or use moesched_bvn_decompose with your own scratch.
+ *
+ * The first call on each device looks up the array's device address (no allocation, but
+ * a runtime query): make that first call with the device current and outside any stream
+ * capture. All calls share the one array; it holds whatever the previous call left and is
+ * fully rewritten for the rows it uses, so nothing needs clearing, but two calls that can
+ * run at the same time on one GPU (different streams, threads or processes sharing a
+ * context) would trample each other's working copy: serialise them. No cudaMalloc,
+ * cudaFree or other allocating call is made.
+ */
+#define MOESCHED_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int moesched_bvn_decompose_static(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
+                                  int32_t* d_coef, int32_t* d_count, int32_t* d_aug,
+                                  int32_t* d_status, int64_t* d_work, void* stream);
 
 /* CUDA error code (cudaError_t as int) of the last failed CUDA call made by
  * this library on the calling thread; 0 if none. */

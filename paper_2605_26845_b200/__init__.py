@@ -46,8 +46,8 @@ def load_library():
                                 "(there is no CPU fallback)")
         lib = ctypes.CDLL(LIB_PATH)
         lib.moesched_strerror.restype = ctypes.c_char_p
-        for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval",
-                     "moesched_last_cuda_error"):
+        for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
+                     "moesched_schedule_eval", "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         _lib = lib
@@ -154,6 +154,27 @@ def bvn_decompose(demand, k_max=None, want_aug=False, want_work=False, out=None,
                                         _ptr(out.count), _ptr(out.extra), _ptr(scratch), _ptr(out.status),
                                         _ptr(out.work), _stream(dev))
     _check(rc, "moesched_bvn_decompose")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def bvn_decompose_static(demand, out: Schedule) -> Schedule:
+    """BvN decomposition through the entry point that allocates nothing: for callers that may
+    not allocate device memory (a host framework owns the pool, or an allocation would stall a
+    latency-critical loop). `out` must be a complete, caller-made Schedule; the working copy sits
+    in the library's built-in 16 MiB array, so B * N * roundup(N, 8) * 4 must fit in it. Calls
+    that may overlap on one GPU share that array and must be serialised."""
+    lib = load_library()
+    demand = _check_demand(demand)
+    B, N, _ = demand.shape
+    dev = demand.device
+    with torch.cuda.device(dev):
+        rc = lib.moesched_bvn_decompose_static(B, N, _ptr(demand), int(out.perm.shape[1]), _ptr(out.perm),
+                                               _ptr(out.dur), _ptr(out.count), _ptr(out.extra),
+                                               _ptr(out.status), _ptr(out.work), _stream(dev))
+    _check(rc, "moesched_bvn_decompose_static")
     return out
 
 

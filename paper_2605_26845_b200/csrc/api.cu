@@ -4,6 +4,7 @@
 namespace moesched {
 
 static thread_local int g_last_cuda_error = 0;
+int& last_cuda_error_slot() { return g_last_cuda_error; }
 
 // Shared memory one CTA may request on sm_100a (227 KB).
 constexpr size_t SMEM_LIMIT = 227 * 1024;
@@ -110,6 +111,7 @@ const char* moesched_strerror(int code) {
     case MOESCHED_ST_TRUNCATED: return "truncated: the matching budget ran out before the matrix did";
     case MOESCHED_EINVAL: return "invalid argument, or (as a status) input matrix out of range";
     case MOESCHED_ECUDA: return "a CUDA call failed, or (as a status) an internal iteration limit was hit";
+    case MOESCHED_ETOOBIG: return "batch too large for the library's built-in scratch array";
     default: return "unknown moesched code";
   }
 }
