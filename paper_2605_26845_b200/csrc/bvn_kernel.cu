@@ -19,7 +19,7 @@ namespace moesched {
 // to cover every row whose column changed. Returns false when no augmenting path exists
 // (cannot happen for a balanced matrix).
 template <int CPL>
-__device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], int (&mr)[CPL],
+__device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], Match<CPL>& M,
                                              short* x, int& lo, int& hi, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   unsigned F[W], P[W];   // frontier rows; rows met but still below the threshold
@@ -47,8 +47,8 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
         if (any_bit<W>(hit)) {
           visited |= 1u << s;
           par[s] = lowest_bit<W>(hit);
-          if (mr[s] < 0) freeslot = s;
-          else set_bit<W>(met, mr[s]);
+          if (M.mr[s] < 0) freeslot = s;
+          else M.add_to(met, s);
         }
       }
     }
@@ -83,7 +83,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
     const int i = __shfl_sync(FULL, pick<CPL>(par, sl), L);
     const int jprev = x[i];
     __syncwarp();
-    if (lane == L) put<CPL>(mr, sl, i);
+    if (lane == L) M.assign(sl, i);
     if (lane == 0) x[i] = (short)j;
     __syncwarp();
     lo = min(lo, i);
@@ -208,9 +208,8 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
     }
     nnz = __reduce_add_sync(FULL, nnz);
 
-    int mr[CPL];
-#pragma unroll
-    for (int s = 0; s < CPL; ++s) mr[s] = -1;
+    Match<CPL> M;
+    M.reset();
     for (int r = lane; r < N; r += 32) x[r] = -1;
     __syncwarp();
 
@@ -230,12 +229,12 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       for (int it = 0; it < N; ++it) {
         const int f = lowest_bit<W>(freerows);
         if (f < 0) break;
-        if (!augment_from<CPL>(N, lane, f, C, mr, x, lo_changed, hi_changed, work)) { okm = false; break; }
+        if (!augment_from<CPL>(N, lane, f, C, M, x, lo_changed, hi_changed, work)) { okm = false; break; }
         clear_bit<W>(freerows, f);
       }
       if (!okm || any_bit<W>(freerows)) { st_code = MOESCHED_ST_INTERNAL; break; }
       work[WK_SKIP] += lo_changed;
-      if (!canonicalise<CPL>(N, lane, lo_changed, hi_changed, C, mr, x, hist, work)) {
+      if (!canonicalise<CPL>(N, lane, lo_changed, hi_changed, C, M, x, hist, work)) {
         st_code = MOESCHED_ST_INTERNAL;
         break;
       }
@@ -246,7 +245,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       for (int s = 0; s < CPL; ++s) {
         const int c = lane * CPL + s;
         val[s] = INF32;
-        if (c < N) { val[s] = A.row(mr[s])[c]; cmin = min(cmin, val[s]); }
+        if (c < N) { val[s] = A.row(M.mr[s])[c]; cmin = min(cmin, val[s]); }
       }
       cmin = __reduce_min_sync(FULL, cmin);
       lo_changed = N;
@@ -260,10 +259,11 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
         const int c = lane * CPL + s;
         if (c < N) {
           const int nv = val[s] - cmin;
-          A.row(mr[s])[c] = nv;
+          A.row(M.mr[s])[c] = nv;
           if (nv == 0) {
-            clear_bit<W>(C[s], mr[s]);
-            set_bit<W>(gone, mr[s]);
+#pragma unroll
+            for (int w = 0; w < W; ++w) C[s][w] &= ~M.word(s, w);
+            M.add_to(gone, s);
             ++zeroed;
           }
         }
@@ -276,9 +276,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 #pragma unroll
       for (int w = 0; w < W; ++w) freerows[w] = __reduce_or_sync(FULL, gone[w]);
       // unmatch the rows whose entry vanished
-#pragma unroll
-      for (int s = 0; s < CPL; ++s)
-        if (mr[s] >= 0 && test_bit<W>(freerows, mr[s])) mr[s] = -1;
+      M.release(freerows);
       __syncwarp();
       for (int r = lane; r < N; r += 32)
         if (test_bit<W>(freerows, r)) x[r] = -1;

@@ -93,6 +93,80 @@ __device__ __forceinline__ void put(T (&a)[C], int s, T v) {
     if (s == k) a[k] = v;
 }
 
+// one-hot word w of the set {idx}; empty for idx < 0
+__device__ __forceinline__ unsigned onehot_word(int idx, int w) {
+  return (idx >> 5) == w ? 1u << (idx & 31) : 0u;
+}
+template <int W>
+__device__ __forceinline__ bool intersects(const unsigned (&a)[W], const unsigned (&b)[W]) {
+  unsigned o = 0u;
+#pragma unroll
+  for (int k = 0; k < W; ++k) o |= a[k] & b[k];
+  return o != 0u;
+}
+
+// The matching as the lane sees it: mr[s] = row matched to the lane's column s (-1 = none).
+// For up to 4 columns per lane the row is also kept as a one-hot mask, so that "is my row in
+// this set" is two logic operations instead of a variable shift and select per word.
+template <int CPL>
+struct Match {
+  static constexpr int W = CPL;
+  static constexpr bool CACHED = CPL <= 4;
+  int mr[CPL];
+  unsigned oh[CACHED ? CPL : 1][CACHED ? CPL : 1];
+
+  __device__ __forceinline__ void reset() {
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) mr[s] = -1;
+    if constexpr (CACHED) {
+#pragma unroll
+      for (int s = 0; s < CPL; ++s)
+#pragma unroll
+        for (int w = 0; w < W; ++w) oh[s][w] = 0u;
+    }
+  }
+  __device__ __forceinline__ unsigned word(int s, int w) const {   // s, w compile-time after unrolling
+    if constexpr (CACHED) return oh[s][w];
+    else return onehot_word(mr[s], w);
+  }
+  // slot chosen at run time
+  __device__ __forceinline__ void assign(int slot, int row) {
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) {
+      const bool me = s == slot;
+      mr[s] = me ? row : mr[s];
+      if constexpr (CACHED) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) oh[s][w] = me ? onehot_word(row, w) : oh[s][w];
+      }
+    }
+  }
+  __device__ __forceinline__ int row_of(int slot) const { return pick<CPL>(mr, slot); }
+  __device__ __forceinline__ bool in(const unsigned (&set)[CPL], int s) const {
+    unsigned o = 0u;
+#pragma unroll
+    for (int w = 0; w < W; ++w) o |= set[w] & word(s, w);
+    return o != 0u;
+  }
+  __device__ __forceinline__ void add_to(unsigned (&set)[CPL], int s) const {
+#pragma unroll
+    for (int w = 0; w < W; ++w) set[w] |= word(s, w);
+  }
+  // unmatch the columns whose row is in `rows`
+  __device__ __forceinline__ void release(const unsigned (&rows)[CPL]) {
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) {
+      if (in(rows, s)) {
+        mr[s] = -1;
+        if constexpr (CACHED) {
+#pragma unroll
+          for (int w = 0; w < W; ++w) oh[s][w] = 0u;
+        }
+      }
+    }
+  }
+};
+
 // ---- the matrix in shared memory --------------------------------------------------------
 // Rows [0, split) live in this CTA's shared memory, rows [split, N) in the
 // partner CTA of the cluster (far == generic pointer into its shared memory).
@@ -338,15 +412,14 @@ __device__ __forceinline__ void cluster_epilogue() {
 // to a column > c (a suffix OR over the lanes), row i qualifies through column c iff
 // i is adjacent to c, i < mr[c] and i is in gt(c).
 template <int CPL>
-__device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL][CPL], const int (&mr)[CPL],
+__device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL][CPL], const Match<CPL>& M,
                                                unsigned (&cand)[CPL]) {
   constexpr int W = CPL;
   unsigned own[W];
 #pragma unroll
   for (int w = 0; w < W; ++w) own[w] = 0u;
 #pragma unroll
-  for (int s = 0; s < CPL; ++s)
-    if (mr[s] >= 0) set_bit<W>(own, mr[s]);
+  for (int s = 0; s < CPL; ++s) M.add_to(own, s);
   unsigned above[W];   // rows matched to the columns of higher lanes
 #pragma unroll
   for (int w = 0; w < W; ++w) {
@@ -365,11 +438,11 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
 #pragma unroll
   for (int ss = 0; ss < CPL; ++ss) {
     const int s = CPL - 1 - ss;   // from the lane's highest column down, growing gt as we go
-    if (mr[s] >= 0) {
+    if (M.mr[s] >= 0) {
 #pragma unroll
-      for (int w = 0; w < W; ++w) acc[w] |= C[s][w] & above[w] & ~ge_word(mr[s], w);
-      set_bit<W>(above, mr[s]);
+      for (int w = 0; w < W; ++w) acc[w] |= C[s][w] & above[w] & ~ge_word(M.mr[s], w);
     }
+    M.add_to(above, s);
   }
 #pragma unroll
   for (int w = 0; w < W; ++w) cand[w] = __reduce_or_sync(FULL, acc[w]);
@@ -377,12 +450,12 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
 
 template <int CPL>
 __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int last,
-                                             const unsigned (&C)[CPL][CPL], int (&mr)[CPL], short* x,
+                                             const unsigned (&C)[CPL][CPL], Match<CPL>& M, short* x,
                                              unsigned* hist, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   bool ok_all = true;
   unsigned cand[W];
-  candidate_rows<CPL>(lane, C, mr, cand);
+  candidate_rows<CPL>(lane, C, M, cand);
   int from = start;
   for (int guard = 0; guard < N; ++guard) {
     // next row of the window that could move
@@ -395,11 +468,13 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
     const int xi = x[i];
     work[WK_SWEEP]++;
     // backward search from row i among the rows >= i
-    unsigned anc[W], F[W], alive[W];
+    unsigned anc[W], F[W], alive[W], imask[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) { anc[w] = F[w] = 0u; alive[w] = ge_word(i, w); }
-    set_bit<W>(anc, i);
-    set_bit<W>(F, i);
+    for (int w = 0; w < W; ++w) {
+      imask[w] = onehot_word(i, w);
+      anc[w] = F[w] = imask[w];
+      alive[w] = ge_word(i, w);
+    }
     int level = 0;
     if (lane < W) hist[lane] = pick<W>(F, lane);
     for (int it = 0; it < N; ++it) {
@@ -408,7 +483,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       for (int w = 0; w < W; ++w) acc[w] = 0u;
 #pragma unroll
       for (int s = 0; s < CPL; ++s) {
-        if (mr[s] >= 0 && test_bit<W>(F, mr[s])) {
+        if (M.in(F, s)) {
 #pragma unroll
           for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
         }
@@ -432,7 +507,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
 #pragma unroll
     for (int ss = 0; ss < CPL; ++ss) {
       const int s = CPL - 1 - ss;
-      if (mr[s] >= 0 && test_bit<W>(C[s], i) && test_bit<W>(anc, mr[s])) myslot = s;
+      if (intersects<W>(C[s], imask) && M.in(anc, s)) myslot = s;
     }
     unsigned ball = __ballot_sync(FULL, myslot >= 0);
     if (ball == 0u) { ok_all = false; continue; }
@@ -440,7 +515,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
     const int sl = __shfl_sync(FULL, myslot, L);
     const int jstar = L * CPL + sl;
     if (jstar != xi) {
-      int cur = __shfl_sync(FULL, pick<CPL>(mr, sl), L);   // row that gives up column jstar
+      int cur = __shfl_sync(FULL, M.row_of(sl), L);   // row that gives up column jstar
       // level at which that row was reached
       int lvl = 0;
       for (int d = 1; d <= level; ++d) {
@@ -450,31 +525,31 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       if (lvl == 0) ok_all = false;
       // walk towards row i: each row takes the column of its successor on the cycle
       while (lvl > 0) {
-        unsigned Hm[W];
+        unsigned Hm[W], cmask[W];
 #pragma unroll
-        for (int w = 0; w < W; ++w) Hm[w] = hist[(lvl - 1) * W + w];
+        for (int w = 0; w < W; ++w) { Hm[w] = hist[(lvl - 1) * W + w]; cmask[w] = onehot_word(cur, w); }
         int ms = -1;
 #pragma unroll
         for (int ss = 0; ss < CPL; ++ss) {
           const int s = CPL - 1 - ss;
-          if (mr[s] >= 0 && test_bit<W>(Hm, mr[s]) && test_bit<W>(C[s], cur)) ms = s;
+          if (M.in(Hm, s) && intersects<W>(C[s], cmask)) ms = s;
         }
         unsigned b2 = __ballot_sync(FULL, ms >= 0);
         if (b2 == 0u) { ok_all = false; break; }
         const int L2 = __ffs(b2) - 1;
         const int s2 = __shfl_sync(FULL, ms, L2);
-        const int nxt = __shfl_sync(FULL, pick<CPL>(mr, s2), L2);
-        if (lane == L2) put<CPL>(mr, s2, cur);
+        const int nxt = __shfl_sync(FULL, M.row_of(s2), L2);
+        if (lane == L2) M.assign(s2, cur);
         if (lane == 0) x[cur] = (short)(L2 * CPL + s2);
         last = max(last, cur);
         cur = nxt;
         --lvl;
         work[WK_ROT]++;
       }
-      if (lane == L) put<CPL>(mr, sl, i);
+      if (lane == L) M.assign(sl, i);
       if (lane == 0) x[i] = (short)jstar;
       __syncwarp();
-      candidate_rows<CPL>(lane, C, mr, cand);
+      candidate_rows<CPL>(lane, C, M, cand);
     }
   }
   return ok_all;

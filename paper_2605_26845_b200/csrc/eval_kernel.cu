@@ -6,6 +6,8 @@
 // expert batch time; dispatch, compute and combine advance as a three-stage
 // pipeline. Link idleness is obtained from totals: sum_k (N dur_k - s_k) equals
 // N * sum_k dur_k minus all served tokens.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace moesched {
@@ -30,6 +32,29 @@ __device__ __forceinline__ long long matrix_sum(const MatView& M, int N, int lan
   }
   if (any_negative) *any_negative = __any_sync(FULL, neg);
   return warp_sum64(acc);
+}
+
+// The lane's CPL destination bytes of one matching, packed little-endian.
+template <int CPL>
+struct Packed {
+  typename std::conditional<(CPL > 4), unsigned long long, unsigned>::type v;
+};
+template <int CPL>
+__device__ __forceinline__ Packed<CPL> load_dest(const uint8_t* row, int lane, int N, bool packed_ok) {
+  Packed<CPL> p;
+  const uint8_t* src = row + lane * CPL;
+  if (packed_ok) {
+    if constexpr (CPL == 1) p.v = *src;
+    else if constexpr (CPL == 2) p.v = *reinterpret_cast<const unsigned short*>(src);
+    else if constexpr (CPL == 4) p.v = *reinterpret_cast<const unsigned*>(src);
+    else p.v = *reinterpret_cast<const unsigned long long*>(src);
+  } else {
+    p.v = 0;
+#pragma unroll
+    for (int s = 0; s < CPL; ++s)
+      if (lane * CPL + s < N) p.v |= (decltype(p.v))src[s] << (8 * s);
+  }
+  return p;
 }
 
 template <int CPL, bool CLUSTER>
@@ -59,6 +84,8 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   const int32_t* db = dur + (size_t)b * k_stride;
 
   if (!bad) {
+    // one aligned word holds the lane's CPL destinations when rows of the schedule are CPL-aligned
+    const bool packed_ok = (N % CPL == 0) && ((reinterpret_cast<uintptr_t>(pb) & (CPL - 1)) == 0);
     for (int k0 = 0; k0 < K && !bad; k0 += 32) {
       // lane q prepares the transfer time of matching k0+q
       const int kk = k0 + lane;
@@ -67,47 +94,60 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
       const long long t_mine =
           ((long long)dk_mine * model.bytes_per_token * 8 + model.link_gbps - 1) / model.link_gbps;
       const int kend = min(32, K - k0);
-      for (int q = 0; q < kend; ++q) {
-        const int dk = __shfl_sync(FULL, dk_mine, q);
-        const long long t = __shfl_sync(FULL, t_mine, q);
-        const uint8_t* pk = pb + (size_t)(k0 + q) * N;
-        unsigned cols[W];
+      // fetch the lane's destinations of all matchings of the chunk before using any of them:
+      // 32 independent loads in flight instead of one dependent load per matching
+      Packed<CPL> dest[32];
 #pragma unroll
-        for (int w = 0; w < W; ++w) cols[w] = 0u;
-        int g = 0, oob = 0;
+      for (int q = 0; q < 32; ++q) {
+        dest[q].v = 0;
+        if (q < kend && lane * CPL < N) dest[q] = load_dest<CPL>(pb + (size_t)(k0 + q) * N, lane, N, packed_ok);
+      }
 #pragma unroll
-        for (int s = 0; s < CPL; ++s) {
-          const int r = lane * CPL + s;
-          if (r < N) {
-            const int j = pk[r];
-            if (j < N) {
-              set_bit<W>(cols, j);
-              int* p = D.row(r) + j;
-              const int val = *p;
-              const int sv = min(dk, val);
-              *p = val - sv;
-              g = max(g, sv);
-            } else {
-              oob = 1;
+      for (int q = 0; q < 32; ++q) {
+        if (q < kend && !bad) {
+          const int dk = __shfl_sync(FULL, dk_mine, q);
+          const long long t = __shfl_sync(FULL, t_mine, q);
+          unsigned cols[W];
+#pragma unroll
+          for (int w = 0; w < W; ++w) cols[w] = 0u;
+          int g = 0, oob = 0;
+#pragma unroll
+          for (int s = 0; s < CPL; ++s) {
+            const int r = lane * CPL + s;
+            if (r < N) {
+              const int j = (int)((dest[q].v >> (8 * s)) & 0xff);
+              if (j < N) {
+                set_bit<W>(cols, j);
+                int* p = D.row(r) + j;
+                const int val = *p;
+                const int sv = min(dk, val);
+                *p = val - sv;
+                g = max(g, sv);
+              } else {
+                oob = 1;
+              }
             }
           }
-        }
-        int seen = 0;
+          int seen = 0;
 #pragma unroll
-        for (int w = 0; w < W; ++w) seen += __popc(__reduce_or_sync(FULL, cols[w]));
-        if (__any_sync(FULL, oob) || seen != N) { bad = 1; break; }
-        g = __reduce_max_sync(FULL, g);
-        const long long comp =
-            g > 0 ? model.expert_fixed_ns + ((long long)g * model.expert_ps_per_token + 999) / 1000 : 0;
-        const long long leg = model.reconfig_ns + t;
-        dsp += leg;
-        if (k0 + q == 0) dsp1 = dsp;
-        cmp = max(dsp, cmp) + comp;
-        cmb = max(cmp, cmb) + leg;
-        ser += 2 * leg + comp;
-        comp_sum += comp;
-        dur_sum += dk;
-        __syncwarp();
+          for (int w = 0; w < W; ++w) seen += __popc(__reduce_or_sync(FULL, cols[w]));
+          if (__any_sync(FULL, oob) || seen != N) {
+            bad = 1;
+          } else {
+            g = __reduce_max_sync(FULL, g);
+            const long long comp =
+                g > 0 ? model.expert_fixed_ns + ((long long)g * model.expert_ps_per_token + 999) / 1000 : 0;
+            const long long leg = model.reconfig_ns + t;
+            dsp += leg;
+            if (k0 + q == 0) dsp1 = dsp;
+            cmp = max(dsp, cmp) + comp;
+            cmb = max(cmp, cmb) + leg;
+            ser += 2 * leg + comp;
+            comp_sum += comp;
+            dur_sum += dk;
+          }
+          __syncwarp();
+        }
       }
     }
     if (dur_sum > (1LL << 40)) bad = 1;

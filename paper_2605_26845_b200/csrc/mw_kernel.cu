@@ -13,7 +13,7 @@ namespace moesched {
 template <int CPL>
 struct MwState {
   int v[CPL];     // column duals of the cost problem
-  int mr[CPL];    // row assigned to the lane's column, -1 if free
+  Match<CPL> M;   // row assigned to each of the lane's columns
 };
 
 // One assignment problem. The column duals v carry over from the previous greedy step
@@ -35,7 +35,8 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
       if (lane * CPL + s < N) vmax = max(vmax, st.v[s]);
     vmax = __reduce_max_sync(FULL, vmax);
 #pragma unroll
-    for (int s = 0; s < CPL; ++s) { st.v[s] -= vmax; st.mr[s] = -1; }
+    for (int s = 0; s < CPL; ++s) st.v[s] -= vmax;
+    st.M.reset();
   }
   for (int r = lane; r < N; r += 32) x[r] = -1;
   unsigned freerows[W];
@@ -56,9 +57,9 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
     const unsigned ball = __ballot_sync(FULL, lmin == u);
     const int L = __ffs(ball) - 1;
     const int sl = __shfl_sync(FULL, lslot, L);
-    const int owner = __shfl_sync(FULL, pick<CPL>(st.mr, sl), L);
+    const int owner = __shfl_sync(FULL, st.M.row_of(sl), L);
     if (owner < 0) {
-      if (lane == L) put<CPL>(st.mr, sl, r);
+      if (lane == L) st.M.assign(sl, r);
       if (lane == 0) x[r] = (short)(L * CPL + sl);
     } else {
       set_bit<W>(freerows, r);
@@ -97,7 +98,7 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
       const int L = __ffs(ball) - 1;
       const int sl = __shfl_sync(FULL, lslot, L);
       if (lane == L) scanned |= 1u << sl;
-      const int i = __shfl_sync(FULL, pick<CPL>(st.mr, sl), L);
+      const int i = __shfl_sync(FULL, st.M.row_of(sl), L);
       work[WK_SCAN]++;
       if (i < 0) { jfin = L * CPL + sl; break; }
       const int vj = __shfl_sync(FULL, pick<CPL>(st.v, sl), L);
@@ -123,7 +124,7 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
       const int i = __shfl_sync(FULL, pick<CPL>(pred, sl), L);
       const int jprev = x[i];
       __syncwarp();
-      if (lane == L) put<CPL>(st.mr, sl, i);
+      if (lane == L) st.M.assign(sl, i);
       if (lane == 0) x[i] = (short)j;
       __syncwarp();
       if (i == f) break;
@@ -186,7 +187,8 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
   if (st_code == MOESCHED_ST_OK) {
     MwState<CPL> st;
 #pragma unroll
-    for (int s = 0; s < CPL; ++s) { st.v[s] = 0; st.mr[s] = -1; }
+    for (int s = 0; s < CPL; ++s) st.v[s] = 0;
+    st.M.reset();
     uint8_t* pout = perm + (size_t)b * k_max * N;
     int32_t* dout = dur + (size_t)b * k_max;
     while (k < k_max && nnz > 0) {
@@ -216,14 +218,14 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
             if (red[s] == u && lane * CPL + s < N) C[s][w] |= 1u << q;
         }
       }
-      if (!canonicalise<CPL>(N, lane, 0, N - 1, C, st.mr, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      if (!canonicalise<CPL>(N, lane, 0, N - 1, C, st.M, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
       // serve: the heaviest matched pair sets the duration; matched entries are sent whole
       int dmax = 0, served = 0;
 #pragma unroll
       for (int s = 0; s < CPL; ++s) {
         const int c = lane * CPL + s;
-        if (c < N && st.mr[s] >= 0) {
-          int* p = R.row(st.mr[s]) + c;
+        if (c < N && st.M.mr[s] >= 0) {
+          int* p = R.row(st.M.mr[s]) + c;
           const int val = *p;
           dmax = max(dmax, val);
           served += val != 0;
