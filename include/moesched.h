@@ -218,6 +218,16 @@ int moesched_bvn_decompose_static(int B, int N, const int32_t* d_demand, int k_m
                                   int32_t* d_coef, int32_t* d_count, int32_t* d_aug,
                                   int32_t* d_status, int64_t* d_work, void* stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): enqueue a kernel of `blocks` CTAs of 256
+ * threads, each thread running 8 independent chains of add / min / xor for `iters`
+ * iterations, and return the number of integer lane-operations it executes
+ * (blocks * 256 * iters * 24), or a negative MOESCHED_* code. Timing the launch gives the
+ * integer issue rate the decomposition kernels are measured against. d_out: device,
+ * blocks * 256 uint32 (written so that the work cannot be optimised away).
+ */
+long long moesched_probe_int_ops(int blocks, int iters, uint32_t* d_out, void* stream);
+
 /* CUDA error code (cudaError_t as int) of the last failed CUDA call made by
  * this library on the calling thread; 0 if none. */
 int moesched_last_cuda_error(void);

@@ -50,6 +50,7 @@ def load_library():
                      "moesched_schedule_eval", "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
+        lib.moesched_probe_int_ops.restype = ctypes.c_longlong
         _lib = lib
     return _lib
 
@@ -176,6 +177,25 @@ def bvn_decompose_static(demand, out: Schedule) -> Schedule:
                                                _ptr(out.status), _ptr(out.work), _stream(dev))
     _check(rc, "moesched_bvn_decompose_static")
     return out
+
+
+def probe_int_rate(device=None, blocks=148 * 8, iters=20000, reps=3) -> float:
+    """Measured integer lane-operations per second of the GPU (add / min / logic mix)."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    out = torch.empty(blocks * 256, dtype=torch.int32, device=dev)
+    best = 0.0
+    with torch.cuda.device(dev):
+        for _ in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ops = lib.moesched_probe_int_ops(blocks, iters, _ptr(out), _stream(dev))
+            e1.record()
+            if ops < 0:
+                _check(int(ops), "moesched_probe_int_ops")
+            e1.synchronize()
+            best = max(best, ops / (e0.elapsed_time(e1) * 1e-3))
+    return best
 
 
 SCORE_FIELDS = ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",
