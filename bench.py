@@ -100,6 +100,26 @@ def measured_peaks():
     return {"hbm_gbs": FALLBACK_HBM_GBS, "sm_max_mhz": 1965.0}, "fallback"
 
 
+def captured_traffic(name):
+    """DRAM bytes per launch from the committed ncu capture, or None once the kernel's source has
+    changed since the counters were taken."""
+    import hashlib
+    src = {"bvn_decompose": "bvn_kernel.cu", "mw_decompose": "mw_kernel.cu", "schedule_eval(bvn)": "eval_kernel.cu"}
+    path = os.path.join(ROOT, "profiles", "dram_traffic_config3.txt")
+    if name not in src or not os.path.exists(path):
+        return None
+    csrc = os.path.join(ROOT, "paper_2605_26845_b200", "csrc")
+    h = hashlib.sha256()
+    for f in ("common.cuh", src[name]):
+        with open(os.path.join(csrc, f), "rb") as fh:
+            h.update(fh.read())
+    for line in open(path):
+        parts = line.split()
+        if len(parts) == 3 and parts[0] == name:
+            return int(parts[1]) if parts[2] == h.hexdigest()[:16] else None
+    return None
+
+
 def algorithmic_ops(work_mw, work_bvn, N):
     """Integer lane-operations the method itself needs, from the kernels' work counters
     (per column or row touched: a handful of adds / compares / bit operations)."""
@@ -319,7 +339,7 @@ def main():
             "kernels_ms": {n: float(t) for n, t in zip(names, per_kernel)},
             "rates": {"greedy_per_s": B / (per_kernel[0] * 1e-3), "bvn_per_s": B / (per_kernel[2] * 1e-3)},
             "roofline": {"kernel": names[dom], "bound": "alu", "achieved": achieved, "peak": alu_peak,
-                         "unit": "Gop/s", "frac": achieved / alu_peak, "traffic": None,
+                         "unit": "Gop/s", "frac": achieved / alu_peak, "traffic": captured_traffic(names[dom]),
                          "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (sampled)",
                          "peak_measured_int_mix": alu_measured, "frac_of_measured_int_mix": achieved / alu_measured,
                          "hbm_side": {"algorithmic_bytes": bytes_bvn,
