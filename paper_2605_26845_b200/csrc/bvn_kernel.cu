@@ -20,7 +20,8 @@ namespace moesched {
 // (cannot happen for a balanced matrix).
 template <int CPL>
 __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], Match<CPL>& M,
-                                             short* x, int& lo, int& hi, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+                                             short* x, int& lo, int& hi, unsigned (&changed)[CPL],
+                                             unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   unsigned F[W], P[W];   // frontier rows; rows met but still below the threshold
 #pragma unroll
@@ -88,6 +89,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
     __syncwarp();
     lo = min(lo, i);
     hi = max(hi, i);
+    set_bit<W>(changed, i);
     work[WK_AUG]++;
     if (i == f) return true;
     j = jprev;
@@ -106,6 +108,9 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
                                                   long long* __restrict__ work_out) {
   constexpr int W = CPL;
   constexpr bool CLUSTER = MODE == 1;
+  // remembering which rows a search depended on pays off from N > 64 on (measured); below that the
+  // searches are so short that the bookkeeping costs more than the searches it saves
+  constexpr bool USE_MEMO = CPL >= 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   WarpCtx cx;
   if constexpr (MODE == 2) cx = warp_prologue_global<CPL>(B, N, S, demand, scratch, smem_raw);
@@ -210,6 +215,9 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 
     Match<CPL> M;
     M.reset();
+    CanonMemo<CPL> memo;
+    memo.reset();
+    for (int q = lane; q < N * W; q += 32) hist[(N + 1) * W + q] = 0u;   // per-row memo starts empty
     for (int r = lane; r < N; r += 32) x[r] = -1;
     __syncwarp();
 
@@ -229,12 +237,12 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       for (int it = 0; it < N; ++it) {
         const int f = lowest_bit<W>(freerows);
         if (f < 0) break;
-        if (!augment_from<CPL>(N, lane, f, C, M, x, lo_changed, hi_changed, work)) { okm = false; break; }
+        if (!augment_from<CPL>(N, lane, f, C, M, x, lo_changed, hi_changed, memo.changed, work)) { okm = false; break; }
         clear_bit<W>(freerows, f);
       }
       if (!okm || any_bit<W>(freerows)) { st_code = MOESCHED_ST_INTERNAL; break; }
       work[WK_SKIP] += lo_changed;
-      if (!canonicalise<CPL>(N, lane, lo_changed, hi_changed, C, M, x, hist, work)) {
+      if (!canonicalise<CPL, USE_MEMO>(N, lane, lo_changed, hi_changed, C, M, x, hist, memo, work)) {
         st_code = MOESCHED_ST_INTERNAL;
         break;
       }

@@ -288,7 +288,8 @@ __device__ __forceinline__ bool load_rows(int* dst, const int32_t* g, int N, int
 }
 
 // ---- per-warp set-up shared by the kernels ----------------------------------------------------
-// Shared memory of one warp: [matrix rows held here][hist: (N+1)*W words][x: N shorts][mbarrier][flag].
+// Shared memory of one warp: [matrix rows held here][hist: (N+1)*W words of search levels, then N*W
+// words of per-row memo][x: N shorts][mbarrier][flag].
 // In cluster mode the grid has two CTAs (one warp each) per matrix: CTA 0 of the pair
 // works, CTA 1 loads rows [split, N) into its own shared memory and then only keeps
 // them available to CTA 0 (distributed shared memory) until the final cluster barrier.
@@ -303,9 +304,10 @@ struct WarpCtx {
 };
 
 __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
+__host__ __device__ inline size_t hist_bytes_for(int N, int W) { return align16((size_t)(2 * N + 1) * W * 4); }
 __host__ __device__ inline size_t warp_smem_bytes(int N, int S, int W, bool cluster) {
   const int rows_here = cluster ? (N + 1) / 2 : N;
-  return align16((size_t)rows_here * S * 4) + align16((size_t)(N + 1) * W * 4) + align16((size_t)N * 2) + 16;
+  return align16((size_t)rows_here * S * 4) + hist_bytes_for(N, W) + align16((size_t)N * 2) + 16;
 }
 
 template <int CPL, bool CLUSTER>
@@ -318,7 +320,7 @@ __device__ __forceinline__ WarpCtx warp_prologue(int B, int N, int S, const int3
   const int split = CLUSTER ? (N + 1) / 2 : N;
   const int rows_here = CLUSTER ? split : N;
   const size_t mat_bytes = align16((size_t)rows_here * S * 4);
-  const size_t hist_bytes = align16((size_t)(N + 1) * CPL * 4);
+  const size_t hist_bytes = hist_bytes_for(N, CPL);
   const size_t x_bytes = align16((size_t)N * 2);
   unsigned char* base = smem_raw + (size_t)warp * warp_smem_bytes(N, S, CPL, CLUSTER);
   int* mat = reinterpret_cast<int*>(base);
@@ -355,7 +357,7 @@ __device__ __forceinline__ WarpCtx warp_prologue(int B, int N, int S, const int3
 // S ints, one N x S slab per matrix): shared memory then holds only hist and x, so many more
 // warps fit on an SM. Suits kernels that touch the matrix a few times per matching.
 __host__ __device__ inline size_t warp_smem_bytes_global(int N, int W) {
-  return align16((size_t)(N + 1) * W * 4) + align16((size_t)N * 2);
+  return hist_bytes_for(N, W) + align16((size_t)N * 2);
 }
 
 template <int CPL>
@@ -367,7 +369,7 @@ __device__ __forceinline__ WarpCtx warp_prologue_global(int B, int N, int S, con
   const int wpb = blockDim.x >> 5;
   unsigned char* base = smem_raw + (size_t)warp * warp_smem_bytes_global(N, CPL);
   cx.hist = reinterpret_cast<unsigned*>(base);
-  cx.x = reinterpret_cast<short*>(base + align16((size_t)(N + 1) * CPL * 4));
+  cx.x = reinterpret_cast<short*>(base + hist_bytes_for(N, CPL));
   cx.b = blockIdx.x * wpb + warp;
   cx.worker = cx.b < B;
   cx.loaded = true;
@@ -448,20 +450,81 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
   for (int w = 0; w < W; ++w) cand[w] = __reduce_or_sync(FULL, acc[w]);
 }
 
-template <int CPL>
+// Memo carried from one call to the next when the graph only loses edges between calls
+// (Birkhoff): known = rows whose last search found no lower column and whose searched set
+// (the rows that could reach them) is recorded; desc[r] (shared memory, W words per row,
+// after the level history) = rows that have r in their recorded set. Such a row needs no new
+// search until a row of its recorded set changes column: new alternating steps only lead
+// INTO rows that changed, so a row that reaches it through them would have to pass a changed
+// row that already reached it before. changed = rows whose column changed since the last call.
+template <int W>
+struct CanonMemo {
+  unsigned known[W];
+  unsigned changed[W];
+  __device__ __forceinline__ void reset() {
+#pragma unroll
+    for (int w = 0; w < W; ++w) known[w] = changed[w] = 0u;
+  }
+};
+
+// rows recorded as depending on any row of `rows`; their entries are consumed
+template <int W>
+__device__ __forceinline__ void collect_dependants(int N, int lane, const unsigned (&rows)[W], unsigned* desc,
+                                                   unsigned (&out)[W]) {
+  unsigned left[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) left[w] = rows[w];
+  for (int it = 0; it < N; ++it) {
+    const int r = lowest_bit<W>(left);
+    if (r < 0) break;
+    clear_bit<W>(left, r);
+#pragma unroll
+    for (int w = 0; w < W; ++w) out[w] |= desc[r * W + w];
+  }
+  __syncwarp();
+  // lane l clears the entries of the rows l, l+32, ... that were just read
+#pragma unroll
+  for (int k = 0; k < W; ++k) {
+    if ((rows[k] >> lane) & 1u) {
+#pragma unroll
+      for (int w = 0; w < W; ++w) desc[(k * 32 + lane) * W + w] = 0u;
+    }
+  }
+  __syncwarp();
+}
+
+template <int CPL, bool MEMO>
 __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int last,
                                              const unsigned (&C)[CPL][CPL], Match<CPL>& M, short* x,
-                                             unsigned* hist, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+                                             unsigned* hist, CanonMemo<CPL>& memo,
+                                             unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
+  unsigned* desc = hist + (N + 1) * W;
   bool ok_all = true;
-  unsigned cand[W];
+  unsigned cand[W], stale[W];   // stale: rows whose recorded set contains a changed row
+#pragma unroll
+  for (int w = 0; w < W; ++w) stale[w] = 0u;
+  if constexpr (MEMO) {
+    collect_dependants<W>(N, lane, memo.changed, desc, stale);
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      stale[w] |= memo.changed[w];
+      memo.known[w] &= ~stale[w];    // rows before `start` keep their column but lose their record
+      memo.changed[w] = 0u;
+    }
+  }
   candidate_rows<CPL>(lane, C, M, cand);
   int from = start;
   for (int guard = 0; guard < N; ++guard) {
-    // next row of the window that could move
+    // next row that could move and is not covered by a record that still holds:
+    // unrecorded rows up to the last changed row
     unsigned todo[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) todo[w] = cand[w] & ge_word(from, w);
+    for (int w = 0; w < W; ++w) {
+      unsigned need = cand[w] & ge_word(from, w);
+      if constexpr (MEMO) need &= ~memo.known[w] & ~ge_word(last + 1, w);
+      todo[w] = need;
+    }
     const int i = lowest_bit<W>(todo);
     if (i < 0 || i > last) break;
     from = i + 1;
@@ -514,7 +577,17 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
     const int L = __ffs(ball) - 1;
     const int sl = __shfl_sync(FULL, myslot, L);
     const int jstar = L * CPL + sl;
-    if (jstar != xi) {
+    if (jstar == xi) {
+      if constexpr (MEMO) {
+        // record: row i stays put until one of the rows that can reach it changes column
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+          if ((anc[w] >> lane) & 1u) desc[(w * 32 + lane) * W + (i >> 5)] |= 1u << (i & 31);
+          memo.known[w] |= imask[w];
+        }
+        __syncwarp();
+      }
+    } else {
       int cur = __shfl_sync(FULL, M.row_of(sl), L);   // row that gives up column jstar
       // level at which that row was reached
       int lvl = 0;
@@ -523,11 +596,18 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         if ((hw >> (cur & 31)) & 1u) lvl = d;
       }
       if (lvl == 0) ok_all = false;
+      unsigned moved[W];
+#pragma unroll
+      for (int w = 0; w < W; ++w) moved[w] = imask[w];
       // walk towards row i: each row takes the column of its successor on the cycle
       while (lvl > 0) {
         unsigned Hm[W], cmask[W];
 #pragma unroll
-        for (int w = 0; w < W; ++w) { Hm[w] = hist[(lvl - 1) * W + w]; cmask[w] = onehot_word(cur, w); }
+        for (int w = 0; w < W; ++w) {
+          Hm[w] = hist[(lvl - 1) * W + w];
+          cmask[w] = onehot_word(cur, w);
+          moved[w] |= cmask[w];
+        }
         int ms = -1;
 #pragma unroll
         for (int ss = 0; ss < CPL; ++ss) {
@@ -549,6 +629,15 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       if (lane == L) M.assign(sl, i);
       if (lane == 0) x[i] = (short)jstar;
       __syncwarp();
+      if constexpr (MEMO) {
+        // the moved rows changed column: every record that contains one of them is void
+        unsigned hit[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) hit[w] = moved[w];
+        collect_dependants<W>(N, lane, moved, desc, hit);
+#pragma unroll
+        for (int w = 0; w < W; ++w) memo.known[w] &= ~hit[w];
+      }
       candidate_rows<CPL>(lane, C, M, cand);
     }
   }

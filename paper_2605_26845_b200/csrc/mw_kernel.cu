@@ -218,7 +218,12 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
             if (red[s] == u && lane * CPL + s < N) C[s][w] |= 1u << q;
         }
       }
-      if (!canonicalise<CPL>(N, lane, 0, N - 1, C, st.M, x, hist, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      CanonMemo<CPL> memo;   // unused: every greedy step has a new graph
+      memo.reset();
+      if (!canonicalise<CPL, false>(N, lane, 0, N - 1, C, st.M, x, hist, memo, work)) {
+        st_code = MOESCHED_ST_INTERNAL;
+        break;
+      }
       // serve: the heaviest matched pair sets the duration; matched entries are sent whole
       int dmax = 0, served = 0;
 #pragma unroll
