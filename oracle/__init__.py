@@ -15,7 +15,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "moesched_oracle.cpp")
 _SO = os.path.join(_HERE, "libmoesched_oracle.so")
 
-MODEL_FIELDS = ("bytes_per_token", "link_gbps", "reconfig_ns", "expert_fixed_ns", "expert_ps_per_token")
+MODEL_FIELDS = ("bytes_per_token", "link_gbps", "reconfig_ns", "expert_fixed_ns", "expert_ps_per_token",
+                "expert_knee_tokens")
 
 
 def build(force: bool = False) -> str:
@@ -82,7 +83,7 @@ def schedule_eval(demand, perm, dur, count, model, threads=1):
     dur = np.ascontiguousarray(dur, dtype=np.int32)
     count = np.ascontiguousarray(count, dtype=np.int32)
     k_stride = perm.shape[1]
-    m = np.array([int(model[f]) for f in MODEL_FIELDS], np.int64)
+    m = np.array([int(model.get(f, 0)) for f in MODEL_FIELDS], np.int64)
     out = {k: np.zeros(B, np.int64) for k in
            ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",
             "unserved_tokens")}
@@ -95,6 +96,18 @@ def schedule_eval(demand, perm, dur, count, model, threads=1):
         raise ValueError("oracle_schedule_eval rejected its arguments")
     out["status"] = status
     return out
+
+
+def ideal_a2a(demand, model):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    m = np.array([int(model.get(f, 0)) for f in MODEL_FIELDS], np.int64)
+    comm = np.zeros(B, np.int64)
+    mk = np.zeros(B, np.int64)
+    status = np.zeros(B, np.int32)
+    if lib().oracle_ideal_a2a(B, N, _p(d), _p(m), _p(comm), _p(mk), _p(status)) != 0:
+        raise ValueError("oracle_ideal_a2a rejected its arguments")
+    return dict(comm_ns=comm, makespan_ns=mk, status=status)
 
 
 def max_weight_perm(W, tier):

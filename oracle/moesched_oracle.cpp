@@ -387,10 +387,19 @@ void bvn_one(int tier, int N, const int32_t* D, int k_max, uint8_t* perm, int32_
 // Schedule scoring [Sec. 4.1 "Execution time"; Sec. 3.3].
 // ---------------------------------------------------------------------------
 struct Model {
-  i64 bytes_per_token, link_gbps, reconfig_ns, expert_fixed_ns, expert_ps_per_token;
+  i64 bytes_per_token, link_gbps, reconfig_ns, expert_fixed_ns, expert_ps_per_token, expert_knee_tokens;
 };
 
 i64 cdiv(i64 x, i64 y) { return (x + y - 1) / y; }
+
+// Time of one expert batch of g tokens on the busiest rank [Sec. 2.2 "Compute time is not
+// strictly linear", Fig. 1]: nothing to do costs nothing; up to the knee the fixed overhead
+// dominates (flat); beyond it the time grows linearly. knee = 0 gives the affine model.
+i64 batch_time(const Model& m, i64 g) {
+  if (g <= 0) return 0;
+  const i64 beyond = g > m.expert_knee_tokens ? g - m.expert_knee_tokens : 0;
+  return m.expert_fixed_ns + cdiv(beyond * m.expert_ps_per_token, 1000);
+}
 
 const i64 DUR_SUM_MAX = 1LL << 40;
 
@@ -426,7 +435,7 @@ void eval_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t
     // matching time = largest transfer / bandwidth (bits / (Gb/s) = ns)
     i64 t = cdiv((i64)dur[k] * m.bytes_per_token * 8, m.link_gbps);
     // ranks compute in parallel: the busiest rank sets the batch time
-    i64 comp = g > 0 ? m.expert_fixed_ns + cdiv(g * m.expert_ps_per_token, 1000) : 0;
+    i64 comp = batch_time(m, g);
     dsp = dsp + m.reconfig_ns + t;               // circuits are set up, then the matching is sent
     if (k == 0) dsp1 = dsp;
     cmp = std::max(dsp, cmp) + comp;             // compute starts when its dispatch has completed
@@ -443,6 +452,11 @@ void eval_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t
   for (size_t e = 0; e < NN; ++e) un += R[e];
   *unserved = un;
   *status = ST_OK;
+}
+
+bool model_ok(const Model& m) {
+  return m.bytes_per_token >= 1 && m.link_gbps >= 1 && m.reconfig_ns >= 0 && m.expert_fixed_ns >= 0 &&
+         m.expert_ps_per_token >= 0 && m.expert_knee_tokens >= 0;
 }
 
 template <class F>
@@ -484,17 +498,15 @@ int oracle_bvn_decompose(int B, int N, const int32_t* demand, int k_max, uint8_t
   return 0;
 }
 
-// model = {bytes_per_token, link_gbps, reconfig_ns, expert_fixed_ns, expert_ps_per_token}
+// model = {bytes_per_token, link_gbps, reconfig_ns, expert_fixed_ns, expert_ps_per_token, expert_knee_tokens}
 int oracle_schedule_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm,
                          const int32_t* dur, const int32_t* count, const int64_t* model,
                          int64_t* overlap_ns, int64_t* serial_ns, int64_t* compute_idle_ns,
                          int64_t* link_idle_tokens, int64_t* unserved_tokens, int32_t* status,
                          int threads) {
   if (B < 0 || N < 1 || N > 256 || k_stride < 1 || !demand || !perm || !dur || !count || !model) return -1;
-  Model m = {model[0], model[1], model[2], model[3], model[4]};
-  if (m.bytes_per_token < 1 || m.link_gbps < 1 || m.reconfig_ns < 0 || m.expert_fixed_ns < 0 ||
-      m.expert_ps_per_token < 0)
-    return -1;
+  Model m = {model[0], model[1], model[2], model[3], model[4], model[5]};
+  if (!model_ok(m)) return -1;
   const size_t NN = (size_t)N * N;
   parallel_for(B, threads, [&](int b) {
     i64 o, s, in, it, un;
@@ -509,6 +521,37 @@ int oracle_schedule_eval(int B, int N, const int32_t* demand, int k_stride, cons
     overlap_ns[b] = o; serial_ns[b] = s; compute_idle_ns[b] = in;
     link_idle_tokens[b] = it; unserved_tokens[b] = un;
   });
+  return 0;
+}
+
+// Idealised congestion-free all-to-all [Sec. 4.1 "Comparisons": "the theoretical completion
+// time for a given communication matrix"]: every port sends and receives at line rate, so the
+// exchange lasts as long as the busiest port (largest row or column sum); like the sequential
+// baseline it runs dispatch, compute and combine to completion one after the other, with all
+// tokens of a rank in one batch and no circuit reconfiguration.
+int oracle_ideal_a2a(int B, int N, const int32_t* demand, const int64_t* model, int64_t* comm_ns,
+                     int64_t* makespan_ns, int32_t* status) {
+  if (B < 0 || N < 1 || N > 256 || !demand || !model) return -1;
+  Model m = {model[0], model[1], model[2], model[3], model[4], model[5]};
+  if (!model_ok(m)) return -1;
+  for (int b = 0; b < B; ++b) {
+    const int32_t* D = demand + (size_t)b * N * N;
+    std::vector<i64> r(N, 0), c(N, 0);
+    bool bad = false;
+    for (int i = 0; i < N; ++i)
+      for (int j = 0; j < N; ++j) {
+        if (D[i * N + j] < 0) bad = true;
+        r[i] += D[i * N + j];
+        c[j] += D[i * N + j];
+      }
+    i64 port = 0, recv = 0;
+    for (int i = 0; i < N; ++i) { port = std::max(port, std::max(r[i], c[i])); recv = std::max(recv, c[i]); }
+    if (bad || port > I32_MAX) { comm_ns[b] = makespan_ns[b] = 0; status[b] = ST_BAD_INPUT; continue; }
+    const i64 t = cdiv(port * m.bytes_per_token * 8, m.link_gbps);
+    comm_ns[b] = t;
+    makespan_ns[b] = 2 * t + batch_time(m, recv);
+    status[b] = ST_OK;
+  }
   return 0;
 }
 

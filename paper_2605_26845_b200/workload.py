@@ -37,7 +37,11 @@ SEED = 260526845
 # hidden size 7168), 400 Gb/s ports, 10 us reconfiguration, expert batch cost
 # 20 us + 0.5 ns per token.
 DEFAULT_MODEL = dict(bytes_per_token=14336, link_gbps=400, reconfig_ns=10_000,
-                     expert_fixed_ns=20_000, expert_ps_per_token=500)
+                     expert_fixed_ns=20_000, expert_ps_per_token=500, expert_knee_tokens=0)
+# The two constants the paper gives for its profiled expert-compute curve (Fig. 1, Sec. 3.1): about
+# 250 us up to about 256 tokens, linear beyond (the slope is not stated; the affine model's is kept),
+# with the 10 ns reconfiguration delay of its evaluation (Sec. 4.1).
+PROFILED_MODEL = dict(DEFAULT_MODEL, reconfig_ns=10, expert_fixed_ns=250_000, expert_knee_tokens=256)
 
 CONFIGS = {
     1: dict(N=8, B=64, tokens=4096, experts=8, top_k=2, kind="zipf", s=1.2, owner="block",

@@ -165,3 +165,59 @@ def test_fragmentation_penalty_trend():
         mv = oracle.schedule_eval(D, v["perm"], v["coef"], v["count"], m)["makespan_overlap_ns"]
         ratios.append(float((mv / mg).mean()))
     assert ratios[0] < ratios[1] < ratios[2] and ratios[2] > 2.0
+
+
+def test_knee_compute_model():
+    """Fig. 1: flat up to the knee, linear beyond; no tokens, no kernel."""
+    from paper_2605_26845_b200.workload import PROFILED_MODEL
+    m = dict(PROFILED_MODEL, reconfig_ns=0, bytes_per_token=1, link_gbps=8)       # 1 token = 1 ns on the link
+    assert m["expert_fixed_ns"] == 250_000 and m["expert_knee_tokens"] == 256
+    for tokens, comp in ((1, 250_000), (256, 250_000), (257, 250_001), (1256, 250_500), (2256, 251_000)):
+        D = np.zeros((1, 4, 4), np.int32)
+        D[0, 1, 2] = tokens
+        perm = np.zeros((1, 1, 4), np.uint8)
+        perm[0, 0] = [0, 2, 1, 3]
+        out = oracle.schedule_eval(D, perm, np.array([[tokens]], np.int32), np.array([1], np.int32), m)
+        assert out["makespan_overlap_ns"][0] == 2 * tokens + comp
+    # knee = 0 is the affine model
+    a = dict(DEFAULT_MODEL)
+    b = dict(DEFAULT_MODEL, expert_knee_tokens=0)
+    D = make_demand(1, 4)
+    s = oracle.mw_decompose(D, 8)
+    ra = oracle.schedule_eval(D, s["perm"], s["dur"], s["count"], a)
+    rb = oracle.schedule_eval(D, s["perm"], s["dur"], s["count"], b)
+    assert (ra["makespan_overlap_ns"] == rb["makespan_overlap_ns"]).all()
+    # with the profiled floor the fragmented BvN schedule pays 250 us per matching (Sec. 4.2)
+    v = oracle.bvn_decompose(D, bvn_capacity(8))
+    rk = oracle.schedule_eval(D, v["perm"], v["coef"], v["count"], PROFILED_MODEL)
+    assert (rk["makespan_serial_ns"] >= 250_000 * v["count"]).all()
+
+
+def test_ideal_all_to_all_bound():
+    m = dict(DEFAULT_MODEL)
+    # uniform matrix: every port carries N*m tokens
+    D = np.full((1, 8, 8), 100, np.int32)
+    out = oracle.ideal_a2a(D, m)
+    t = -(-800 * 14336 * 8 // 400)
+    assert out["comm_ns"][0] == t and out["makespan_ns"][0] == 2 * t + 20_000 + 400
+    # incast: column 0 receives from everybody; the receiving port is the bottleneck
+    D = np.zeros((1, 8, 8), np.int32)
+    D[0, :, 0] = 50
+    out = oracle.ideal_a2a(D, m)
+    assert out["comm_ns"][0] == -(-400 * 14336 * 8 // 400)
+    assert oracle.ideal_a2a(np.zeros((1, 4, 4), np.int32), m)["makespan_ns"][0] == 0
+    neg = np.zeros((1, 4, 4), np.int32)
+    neg[0, 1, 1] = -3
+    assert oracle.ideal_a2a(neg, m)["status"][0] == -1
+    # any complete schedule of matchings needs at least the busiest port's tokens of link time, and
+    # the BvN schedule of the balanced matrix needs exactly that many (its coefficients sum to T)
+    D = make_demand(2, 8)
+    ideal = oracle.ideal_a2a(D, m)
+    g = oracle.mw_decompose(D, 64)
+    v = oracle.bvn_decompose(D, bvn_capacity(16))
+    port = np.maximum(D.sum(1).max(1), D.sum(2).max(1))
+    for b in range(8):
+        assert v["coef"][b, :v["count"][b]].sum() == port[b]
+        assert g["dur"][b, :g["count"][b]].sum() >= port[b]
+        link = sum(-(-int(c) * 14336 * 8 // 400) for c in v["coef"][b, :v["count"][b]])
+        assert ideal["comm_ns"][b] <= link <= ideal["comm_ns"][b] + v["count"][b]
