@@ -284,6 +284,18 @@ def main():
         total_ms += marks[0].elapsed_time(marks[4])
     per_kernel /= args.steps
 
+    # ---- the all-to-all yardstick (not part of the step): one streaming pass over the demand ----
+    a2a_ms = []
+    for _ in range(5):
+        flush.fill_(1)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        ms.ideal_a2a(d, DEFAULT_MODEL)
+        a1.record(stream)
+        a1.synchronize()
+        a2a_ms.append(a0.elapsed_time(a1))
+    a2a_ms = float(np.median(a2a_ms))
+
     # ---- end to end: pinned host demand in, schedules and scores back to pinned host memory ----
     h_in = torch.from_numpy(D_host).pin_memory()
     outs = [mw.perm, mw.dur, mw.count, mw.status, bv.perm, bv.dur, bv.count, bv.status, score_mw, score_bv]
@@ -345,6 +357,10 @@ def main():
                          "hbm_side": {"algorithmic_bytes": bytes_bvn,
                                       "gbs": bytes_bvn / (per_kernel[2] * 1e-3) / 1e9,
                                       "peak_gbs": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}"}},
+            "ideal_a2a_kernel": {"ms": a2a_ms, "bound": "hbm", "achieved": 4.0 * B * N * N / (a2a_ms * 1e-3) / 1e9,
+                                 "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": 4.0 * B * N * N / (a2a_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                 "peak_kind": f"of {peak_kind}"},
             "e2e": {"value": aggregate_value(world, B, e2e_steps, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": 4 * args.steps,

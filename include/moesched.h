@@ -70,13 +70,19 @@ extern "C" {
  * expert batch costs a fixed overhead plus a per-token cost (the affine form
  * of the "knee" of Fig. 1); circuits are reconfigured before every matching.
  * All integers. Ranges: 1 <= bytes_per_token <= 2^20, 1 <= link_gbps <= 2^20,
- * 0 <= reconfig_ns, expert_fixed_ns <= 2^40, 0 <= expert_ps_per_token <= 2^30. */
+ * 0 <= reconfig_ns, expert_fixed_ns <= 2^40, 0 <= expert_ps_per_token <= 2^30,
+ * 0 <= expert_knee_tokens <= 2^31-1.
+ * Batch time of g > 0 tokens: expert_fixed_ns + ceil(max(0, g - expert_knee_tokens) *
+ * expert_ps_per_token / 1000); 0 for g = 0. expert_knee_tokens = 0 is the affine model;
+ * 250000 ns with a knee of 256 tokens are the constants the paper reports for its profiled
+ * curve (Fig. 1, Sec. 3.1). */
 typedef struct moesched_model {
   int64_t bytes_per_token;     /* payload of one routed token, bytes            */
   int64_t link_gbps;           /* port speed in Gb/s == bits per nanosecond     */
   int64_t reconfig_ns;         /* circuit reconfiguration delay per matching    */
   int64_t expert_fixed_ns;     /* fixed cost of one expert batch                */
   int64_t expert_ps_per_token; /* marginal cost per token, picoseconds          */
+  int64_t expert_knee_tokens;  /* batch size up to which only the fixed cost is paid */
 } moesched_model_t;
 
 /*
@@ -164,7 +170,7 @@ size_t moesched_bvn_scratch_bytes(int B, int N);
  *   served_i = min(dur_k, Dres[i][pi_k(i)]); Dres -= served  (real tokens first)
  *   g_k = max_i served_i, s_k = sum_i served_i
  *   t_k    = ceil(dur_k * bytes_per_token * 8 / link_gbps)            [ns]
- *   comp_k = g_k > 0 ? expert_fixed_ns + ceil(g_k * expert_ps_per_token / 1000) : 0
+ *   comp_k = batch time of g_k tokens (see moesched_model_t)
  *   Dsp_k = Dsp_{k-1} + reconfig_ns + t_k
  *   Cmp_k = max(Dsp_k, Cmp_{k-1}) + comp_k
  *   Cmb_k = max(Cmp_k, Cmb_{k-1}) + reconfig_ns + t_k
@@ -187,6 +193,25 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride,
                            int64_t* d_makespan_serial_ns, int64_t* d_compute_idle_ns,
                            int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
                            int32_t* d_status, void* stream);
+
+/*
+ * Idealised congestion-free all-to-all (paper Sec. 4.1 "Comparisons": "the theoretical
+ * completion time for a given communication matrix"), the yardstick the decomposed
+ * schedules are compared with. Every port sends and receives at line rate, so one exchange
+ * lasts as long as its busiest port; dispatch, expert compute (all tokens of a rank in one
+ * batch) and combine run to completion one after the other; no circuit is reconfigured.
+ *   port_b  = max(largest row sum, largest column sum) of matrix b
+ *   comm_ns = ceil(port_b * bytes_per_token * 8 / link_gbps)
+ *   makespan_ns = 2 * comm_ns + batch time of the largest column sum
+ *
+ *   d_demand       in   [B][N][N] int32, entries >= 0, row and column sums <= 2^31-1
+ *   h_model        in   HOST pointer, read during the call
+ *   d_comm_ns      out  [B] int64
+ *   d_makespan_ns  out  [B] int64
+ *   d_status       out  [B] int32 (OK, or BAD_INPUT with both outputs 0)
+ */
+int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_model_t* h_model,
+                       int64_t* d_comm_ns, int64_t* d_makespan_ns, int32_t* d_status, void* stream);
 
 /*
  * Birkhoff-von Neumann decomposition for callers that cannot allocate device memory.

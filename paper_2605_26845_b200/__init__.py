@@ -14,7 +14,7 @@ from dataclasses import dataclass
 
 import torch
 
-from .workload import DEFAULT_MODEL, bvn_capacity  # noqa: F401  (re-exported)
+from .workload import DEFAULT_MODEL, PROFILED_MODEL, bvn_capacity  # noqa: F401  (re-exported)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmoesched.so")
@@ -31,7 +31,7 @@ class MoeschedError(RuntimeError):
 class _Model(ctypes.Structure):
     _fields_ = [("bytes_per_token", ctypes.c_int64), ("link_gbps", ctypes.c_int64),
                 ("reconfig_ns", ctypes.c_int64), ("expert_fixed_ns", ctypes.c_int64),
-                ("expert_ps_per_token", ctypes.c_int64)]
+                ("expert_ps_per_token", ctypes.c_int64), ("expert_knee_tokens", ctypes.c_int64)]
 
 
 _lib = None
@@ -47,7 +47,7 @@ def load_library():
         lib = ctypes.CDLL(LIB_PATH)
         lib.moesched_strerror.restype = ctypes.c_char_p
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
-                     "moesched_schedule_eval", "moesched_last_cuda_error"):
+                     "moesched_schedule_eval", "moesched_ideal_a2a", "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         lib.moesched_probe_int_ops.restype = ctypes.c_longlong
@@ -198,6 +198,27 @@ def probe_int_rate(device=None, blocks=148 * 8, iters=20000, reps=3) -> float:
     return best
 
 
+def _model(model):
+    return _Model(**{k: int(v) for k, v in (model or DEFAULT_MODEL).items()})
+
+
+def ideal_a2a(demand, model=None) -> dict:
+    """Idealised congestion-free all-to-all of every matrix: 'comm_ns' (one exchange at line rate of
+    the busiest port), 'makespan_ns' (dispatch + compute + combine, run to completion), 'status'."""
+    lib = load_library()
+    demand = _check_demand(demand)
+    B, N, _ = demand.shape
+    dev = demand.device
+    m = _model(model)
+    out = torch.empty((2, B), dtype=torch.int64, device=dev)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib.moesched_ideal_a2a(B, N, _ptr(demand), ctypes.byref(m), _ptr(out[0]), _ptr(out[1]), _ptr(status),
+                                    _stream(dev))
+    _check(rc, "moesched_ideal_a2a")
+    return {"comm_ns": out[0], "makespan_ns": out[1], "status": status}
+
+
 SCORE_FIELDS = ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", "link_idle_tokens",
                 "unserved_tokens")
 
@@ -213,7 +234,7 @@ def schedule_eval(demand, perm, dur, count, model=None, out=None) -> dict:
     B, N, _ = demand.shape
     if perm.dim() != 3 or perm.shape[0] != B or perm.shape[2] != N or dur.shape != perm.shape[:2]:
         raise MoeschedError("perm must be [B, k_stride, N] and dur [B, k_stride]")
-    m = _Model(**{k: int(v) for k, v in (model or DEFAULT_MODEL).items()})
+    m = _model(model)
     dev = demand.device
     scores = out if out is not None else torch.empty((5, B), dtype=torch.int64, device=dev)
     status = torch.empty(B, dtype=torch.int32, device=dev)

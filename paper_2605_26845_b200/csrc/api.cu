@@ -31,6 +31,14 @@ static int fail_cuda(cudaError_t e) {
   return MOESCHED_ECUDA;
 }
 
+bool model_in_range(const moesched_model_t& m) {
+  const int64_t lim20 = 1LL << 20, lim30 = 1LL << 30, lim40 = 1LL << 40;
+  return m.bytes_per_token >= 1 && m.bytes_per_token <= lim20 && m.link_gbps >= 1 && m.link_gbps <= lim20 &&
+         m.reconfig_ns >= 0 && m.reconfig_ns <= lim40 && m.expert_fixed_ns >= 0 && m.expert_fixed_ns <= lim40 &&
+         m.expert_ps_per_token >= 0 && m.expert_ps_per_token <= lim30 && m.expert_knee_tokens >= 0 &&
+         m.expert_knee_tokens <= 2147483647LL;
+}
+
 static bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
 static bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7) == 0; }
 
@@ -87,11 +95,7 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
       !aligned8(d_link_idle_tokens) || !aligned8(d_unserved_tokens))
     return MOESCHED_EINVAL;
   const moesched_model_t m = *h_model;
-  const int64_t lim20 = 1LL << 20, lim30 = 1LL << 30, lim40 = 1LL << 40;
-  if (m.bytes_per_token < 1 || m.bytes_per_token > lim20 || m.link_gbps < 1 || m.link_gbps > lim20 ||
-      m.reconfig_ns < 0 || m.reconfig_ns > lim40 || m.expert_fixed_ns < 0 || m.expert_fixed_ns > lim40 ||
-      m.expert_ps_per_token < 0 || m.expert_ps_per_token > lim30)
-    return MOESCHED_EINVAL;
+  if (!model_in_range(m)) return MOESCHED_EINVAL;
   if (B == 0) return MOESCHED_OK;
   cudaError_t e = run_eval(B, N, d_demand, k_stride, d_perm, d_dur, d_count, m,
                            reinterpret_cast<long long*>(d_makespan_overlap_ns),
@@ -100,6 +104,21 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
                            reinterpret_cast<long long*>(d_link_idle_tokens),
                            reinterpret_cast<long long*>(d_unserved_tokens), d_status,
                            static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_model_t* h_model, int64_t* d_comm_ns,
+                       int64_t* d_makespan_ns, int32_t* d_status, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N) return MOESCHED_EINVAL;
+  if (!d_demand || !h_model || !d_comm_ns || !d_makespan_ns || !d_status) return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_status) || !aligned8(d_comm_ns) || !aligned8(d_makespan_ns))
+    return MOESCHED_EINVAL;
+  const moesched_model_t m = *h_model;
+  if (!model_in_range(m)) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  cudaError_t e = run_ideal_a2a(B, N, d_demand, m, reinterpret_cast<long long*>(d_comm_ns),
+                                reinterpret_cast<long long*>(d_makespan_ns), d_status,
+                                static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }
 

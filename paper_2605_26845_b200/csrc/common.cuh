@@ -644,6 +644,13 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
   return ok_all;
 }
 
+// Time of one expert batch of g tokens (see moesched_model_t).
+__device__ __forceinline__ long long batch_time_ns(const moesched_model_t& m, long long g) {
+  if (g <= 0) return 0;
+  const long long beyond = g > m.expert_knee_tokens ? g - m.expert_knee_tokens : 0;
+  return m.expert_fixed_ns + (beyond * m.expert_ps_per_token + 999) / 1000;
+}
+
 // ---- host-side launch geometry ---------------------------------------------------------------
 struct Geometry {
   int cpl;       // columns per lane: 1, 2, 4 or 8
@@ -664,6 +671,10 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                      cudaStream_t stream);
+
+bool model_in_range(const moesched_model_t& m);
+cudaError_t run_ideal_a2a(int B, int N, const int32_t* demand, const moesched_model_t& model, long long* comm_ns,
+                          long long* makespan_ns, int32_t* status, cudaStream_t stream);
 
 // Launch helper shared by the three kernels.
 template <typename Kernel, typename... Args>

@@ -135,8 +135,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
             bad = 1;
           } else {
             g = __reduce_max_sync(FULL, g);
-            const long long comp =
-                g > 0 ? model.expert_fixed_ns + ((long long)g * model.expert_ps_per_token + 999) / 1000 : 0;
+            const long long comp = batch_time_ns(model, g);
             const long long leg = model.reconfig_ns + t;
             dsp += leg;
             if (k0 + q == 0) dsp1 = dsp;

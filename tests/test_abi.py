@@ -26,7 +26,7 @@ def declared_functions():
 
 def test_header_declares_the_entry_points():
     names = declared_functions()
-    for want in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval",
+    for want in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval", "moesched_ideal_a2a",
                  "moesched_strerror", "moesched_last_cuda_error"):
         assert want in names
 
@@ -47,6 +47,7 @@ def test_argument_validation_needs_no_gpu(lib):
     assert lib.moesched_bvn_scratch_bytes(1, 300) == 0
     assert lib.moesched_schedule_eval(1, 8, null, 1, null, null, null, null, null, null, null, null, null,
                                       null, null) == -1
+    assert lib.moesched_ideal_a2a(1, 8, null, null, null, null, null, null) == -1
     assert lib.moesched_strerror(0) == b"ok"
     assert lib.moesched_last_cuda_error() == 0
 

@@ -176,3 +176,20 @@ def test_bvn_at_full_size(cfg):
         s2 = ms.bvn_decompose(d, cap, scratch=False)
         kk = used(s)
         assert (s2.count == s.count).all() and (s2.perm[kk] == s.perm[kk]).all() and (s2.dur[kk] == s.dur[kk]).all()
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_ideal_all_to_all_at_full_size(cfg):
+    from paper_2605_26845_b200.workload import PROFILED_MODEL
+    D, d = demand(cfg)
+    for model in (DEFAULT_MODEL, PROFILED_MODEL):
+        got = ms.ideal_a2a(d, model)
+        ref = oracle.ideal_a2a(D, model)                               # cheap: every matrix
+        for name in ("comm_ns", "makespan_ns", "status"):
+            assert (got[name].cpu().numpy() == ref[name]).all(), name
+    # no schedule of matchings can move the busiest port's tokens in less link time
+    s = ms.mw_decompose(d, 4 * D.shape[1])
+    complete = s.status == 0
+    total = torch.where(used(s), s.dur, torch.zeros_like(s.dur)).sum(1).to(torch.int64)
+    port = torch.maximum(d.sum(1).max(1).values, d.sum(2).max(1).values)
+    assert (total[complete] >= port[complete]).all()

@@ -139,3 +139,31 @@ def test_runs_are_deterministic_and_stream_ordered():
     assert (a.count == b.count).all() and (a.status == b.status).all()
     kk = (torch.arange(a.perm.shape[1], device="cuda")[None, :] < a.count[:, None])
     assert (a.perm[kk] == b.perm[kk]).all() and (a.dur[kk] == b.dur[kk]).all()
+
+
+@pytest.mark.parametrize("N", [1, 5, 16, 33, 64, 100, 256])
+def test_ideal_all_to_all_and_knee_model(N):
+    from paper_2605_26845_b200.workload import PROFILED_MODEL
+    D = random_matrices(6, N, seed=4000 + N, kind="uniform", high=3000, zero_frac=0.3)
+    D[1] = 0
+    D[2, 0, 0] = -1
+    d = dev(D)
+    for model in (DEFAULT_MODEL, PROFILED_MODEL, dict(PROFILED_MODEL, expert_knee_tokens=50, expert_fixed_ns=7)):
+        got = ms.ideal_a2a(d, model)
+        ref = oracle.ideal_a2a(D, model)
+        for name in ("comm_ns", "makespan_ns", "status"):
+            assert (got[name].cpu().numpy() == ref[name]).all(), name
+        D2 = D.copy()
+        D2[2, 0, 0] = 1
+        check_all(D2, 4, 6, model=model)              # the knee enters the scores of both schedules
+
+
+def test_ideal_all_to_all_rejects_port_overflow():
+    D = np.zeros((2, 4, 4), np.int32)
+    D[0, 0, :2] = 2**30                               # row sum 2^31: beyond the port range
+    D[1, 0, 0] = 2**31 - 1
+    got = ms.ideal_a2a(dev(D), DEFAULT_MODEL)
+    ref = oracle.ideal_a2a(D, DEFAULT_MODEL)
+    assert list(ref["status"]) == [-1, 0]
+    for name in ("comm_ns", "makespan_ns", "status"):
+        assert (got[name].cpu().numpy() == ref[name]).all(), name
