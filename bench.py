@@ -214,6 +214,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="matrices per GPU (default: the configuration's B)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--overlap", action="store_true",
+                    help="fork greedy and BvN onto two streams (measured slower than one stream)")
     ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS),
                     help="workload configuration (default 3: N=64, the one the metric is quoted on)")
     args = ap.parse_args()
@@ -248,22 +250,25 @@ def main():
     d = torch.from_numpy(D_host).to(dev)
     stream = torch.cuda.current_stream()
 
-    def sched(kcap):
-        return ms.Schedule(perm=torch.empty((B, kcap, N), dtype=torch.uint8, device=dev),
-                           dur=torch.empty((B, kcap), dtype=torch.int32, device=dev),
-                           count=torch.empty(B, dtype=torch.int32, device=dev),
-                           status=torch.empty(B, dtype=torch.int32, device=dev),
-                           work=torch.zeros((B, ms.WORK_FIELDS), dtype=torch.int64, device=dev))
-
-    mw, bv = sched(K_MW), sched(cap)
-    score_mw = torch.empty((5, B), dtype=torch.int64, device=dev)
-    score_bv = torch.empty((5, B), dtype=torch.int64, device=dev)
+    path = ms.Path(B, N, K_MW, cap, device=dev, want_work=True)
+    mw, bv = path.mw, path.bvn
+    score_mw, score_bv, scratch = path.score_mw, path.score_bvn, path.scratch
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-    scratch = torch.empty(ms.bvn_scratch_bytes(B, N), dtype=torch.uint8, device=dev)
 
     names = ["mw_decompose", "schedule_eval(mw)", "bvn_decompose", "schedule_eval(bvn)"]
 
     def step(events=None):
+        """The whole path as a user runs it (ms.Path): four launches on the current stream."""
+        if events is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        path.run(d, DEFAULT_MODEL, overlap=args.overlap)
+        if events is not None:
+            e1.record(stream)
+            events.append((e0, e1))
+
+    def serial_step(events=None):
+        """The same four launches one after the other on one stream: per-kernel durations."""
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)] if events is not None else None
         if marks: marks[0].record(stream)
         ms.mw_decompose(d, K_MW, out=mw)
@@ -294,12 +299,18 @@ def main():
             flush.fill_(1)
             step(events)
         barrier()
+    total_ms = sum(e0.elapsed_time(e1) for e0, e1 in events)
+
+    # ---- per-kernel durations (for the roofline): the same launches, serial, same flush ----
+    kev = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        serial_step(kev)
+    barrier()
     per_kernel = np.zeros(4)
-    total_ms = 0.0
-    for marks in events:
+    for marks in kev:
         for i in range(4):
             per_kernel[i] += marks[i].elapsed_time(marks[i + 1])
-        total_ms += marks[0].elapsed_time(marks[4])
     per_kernel /= args.steps
 
     # ---- the all-to-all yardstick (not part of the step): one streaming pass over the demand ----
@@ -316,7 +327,7 @@ def main():
 
     # ---- end to end: pinned host demand in, schedules and scores back to pinned host memory ----
     h_in = torch.from_numpy(D_host).pin_memory()
-    outs = [mw.perm, mw.dur, mw.count, mw.status, bv.perm, bv.dur, bv.count, bv.status, score_mw, score_bv]
+    outs = path.outputs()
     h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
     h2d = h_in.numel() * h_in.element_size()
     d2h = sum(t.numel() * t.element_size() for t in outs)
@@ -365,8 +376,10 @@ def main():
             "vs_baseline": None, "dtype": "int32", "data": "synthetic",
             "config": {"workload": workload_name(B), "l2": "flushed between timed steps (256 MiB write, untimed)",
                        "matchings_per_matrix": {"greedy": k_mw, "bvn": k_bv}, "all_status_ok": ok,
+                       "streams": "greedy and BvN forked on two streams, joined" if args.overlap else "one",
                        "seed": SEED},
             "kernels_ms": {n: float(t) for n, t in zip(names, per_kernel)},
+            "kernels_ms_note": "per-kernel events from a second, identical serial pass",
             "rates": {"greedy_per_s": B / (per_kernel[0] * 1e-3), "bvn_per_s": B / (per_kernel[2] * 1e-3)},
             "roofline": {"kernel": names[dom], "bound": "alu", "achieved": achieved, "peak": alu_peak,
                          "unit": "Gop/s", "frac": achieved / alu_peak, "traffic": captured_traffic(names[dom]) if CFG == 3 else None,

@@ -167,3 +167,26 @@ def test_ideal_all_to_all_rejects_port_overflow():
     assert list(ref["status"]) == [-1, 0]
     for name in ("comm_ns", "makespan_ns", "status"):
         assert (got[name].cpu().numpy() == ref[name]).all(), name
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+def test_path_runner_matches_separate_calls(overlap):
+    D = make_demand(2, 96)
+    d = dev(D)
+    N = D.shape[1]
+    path = ms.Path(96, N, 16)
+    for _ in range(2):                                   # buffers are reused from run to run
+        path.run(d, DEFAULT_MODEL, overlap=overlap)
+    torch.cuda.current_stream().synchronize()
+    g = ms.mw_decompose(d, 16)
+    v = ms.bvn_decompose(d)
+    for a, b in ((path.mw, g), (path.bvn, v)):
+        kk = torch.arange(a.perm.shape[1], device="cuda")[None, :] < b.count[:, None]
+        assert (a.count == b.count).all() and (a.status == b.status).all()
+        assert (a.perm[kk] == b.perm[kk]).all() and (a.dur[kk] == b.dur[kk]).all()
+    sg = ms.schedule_eval(d, g.perm, g.dur, g.count)
+    sv = ms.schedule_eval(d, v.perm, v.dur, v.count)
+    for i, name in enumerate(ms.SCORE_FIELDS):
+        assert (path.score_mw[i] == sg[name]).all() and (path.score_bvn[i] == sv[name]).all()
+    ref = oracle.schedule_eval(D, g.perm.cpu().numpy(), g.dur.cpu().numpy(), g.count.cpu().numpy(), DEFAULT_MODEL)
+    assert (path.score_mw[0].cpu().numpy() == ref["makespan_overlap_ns"]).all()
