@@ -27,7 +27,8 @@
  *     matching allows, then row 1, ...). Results are therefore unique and
  *     independent of the solver.
  *   - Return value: MOESCHED_OK when the work was enqueued; MOESCHED_EINVAL
- *     for a null pointer or an out-of-range size (nothing enqueued);
+ *     for a null pointer or an out-of-range size (nothing enqueued); B = 0 is
+ *     accepted, enqueues nothing and does not look at the pointers;
  *     MOESCHED_ECUDA when a CUDA call failed (moesched_last_cuda_error()).
  *   - Per-matrix outcome in d_status[b]:
  *       MOESCHED_ST_OK          complete result

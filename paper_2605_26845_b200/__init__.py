@@ -311,3 +311,53 @@ class Path:
         for done in self._join:
             cur.wait_event(done)
         return self
+
+
+class HostPipeline:
+    """The whole path for batches that live in host memory, double-buffered.
+
+    submit() enqueues, for one batch: the copy of the demand from (pinned) host memory to the device
+    on an upload stream, the four kernels on a compute stream, and the copy of all schedules and scores
+    back to pinned host memory on a download stream. With two slots the download of one batch and the
+    upload of the next overlap the kernels of the batch in between, so a stream of batches runs at the
+    speed of the slowest of the three stages instead of their sum."""
+
+    def __init__(self, B, N, k_mw, k_bvn=None, device=None, slots=2):
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.device, self.slots = dev, slots
+        self.paths = [Path(B, N, k_mw, k_bvn, device=dev) for _ in range(slots)]
+        self.d_in = [torch.empty((B, N, N), dtype=torch.int32, device=dev) for _ in range(slots)]
+        self.h_out = [[torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in p.outputs()] for p in self.paths]
+        self.up, self.compute, self.down = (torch.cuda.Stream(dev) for _ in range(3))
+        self.ev_in = [torch.cuda.Event() for _ in range(slots)]
+        self.ev_done = [torch.cuda.Event() for _ in range(slots)]
+        self.ev_out = [torch.cuda.Event() for _ in range(slots)]
+        self._next = 0
+        self.h2d_bytes = B * N * N * 4
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.paths[0].outputs())
+
+    def submit(self, demand_host, model=None) -> int:
+        """Enqueue one batch (a [B, N, N] int32 CPU tensor, ideally pinned); returns its slot."""
+        s = self._next
+        self._next = (s + 1) % self.slots
+        self.ev_out[s].synchronize()            # the slot's previous results must have left the device
+        self.up.wait_event(self.ev_done[s])     # and its previous kernels must be done with the input
+        with torch.cuda.stream(self.up):
+            self.d_in[s].copy_(demand_host, non_blocking=True)
+            self.ev_in[s].record(self.up)
+        self.compute.wait_event(self.ev_in[s])
+        with torch.cuda.stream(self.compute):
+            self.paths[s].run(self.d_in[s], model)
+            self.ev_done[s].record(self.compute)
+        self.down.wait_event(self.ev_done[s])
+        with torch.cuda.stream(self.down):
+            for h, t in zip(self.h_out[s], self.paths[s].outputs()):
+                h.copy_(t, non_blocking=True)
+            self.ev_out[s].record(self.down)
+        return s
+
+    def result(self, slot):
+        """Block until the slot's results are in host memory; returns the pinned host tensors in the
+        order of Path.outputs(). They are overwritten when the slot is submitted again."""
+        self.ev_out[slot].synchronize()
+        return self.h_out[slot]

@@ -52,11 +52,11 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
                           int32_t* d_count, int32_t* d_residual, int32_t* d_status, int64_t* d_work,
                           void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
   if (!d_demand || !d_perm || !d_dur || !d_count || !d_status) return MOESCHED_EINVAL;
   if (!aligned4(d_demand) || !aligned4(d_dur) || !aligned4(d_count) || !aligned4(d_status) ||
       !aligned4(d_residual) || !aligned8(d_work))
     return MOESCHED_EINVAL;
-  if (B == 0) return MOESCHED_OK;
   cudaError_t e = run_mw(B, N, d_demand, k_max, d_perm, d_dur, d_count, d_residual, d_status,
                          reinterpret_cast<long long*>(d_work), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
@@ -71,11 +71,11 @@ int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uin
                            int32_t* d_count, int32_t* d_aug, int32_t* d_scratch, int32_t* d_status,
                            int64_t* d_work, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
   if (!d_demand || !d_perm || !d_coef || !d_count || !d_status) return MOESCHED_EINVAL;
   if (!aligned4(d_demand) || !aligned4(d_coef) || !aligned4(d_count) || !aligned4(d_status) || !aligned4(d_aug) ||
       !aligned8(d_work) || (reinterpret_cast<uintptr_t>(d_scratch) & 31) != 0)
     return MOESCHED_EINVAL;
-  if (B == 0) return MOESCHED_OK;
   cudaError_t e = run_bvn(B, N, d_demand, k_max, d_perm, d_coef, d_count, d_aug, d_scratch, d_status,
                           reinterpret_cast<long long*>(d_work), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
@@ -87,6 +87,7 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
                            int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
                            int32_t* d_status, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_stride < 1) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
   if (!d_demand || !d_perm || !d_dur || !d_count || !h_model || !d_makespan_overlap_ns ||
       !d_makespan_serial_ns || !d_compute_idle_ns || !d_link_idle_tokens || !d_unserved_tokens || !d_status)
     return MOESCHED_EINVAL;
@@ -96,7 +97,6 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
     return MOESCHED_EINVAL;
   const moesched_model_t m = *h_model;
   if (!model_in_range(m)) return MOESCHED_EINVAL;
-  if (B == 0) return MOESCHED_OK;
   cudaError_t e = run_eval(B, N, d_demand, k_stride, d_perm, d_dur, d_count, m,
                            reinterpret_cast<long long*>(d_makespan_overlap_ns),
                            reinterpret_cast<long long*>(d_makespan_serial_ns),
@@ -110,12 +110,12 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
 int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_model_t* h_model, int64_t* d_comm_ns,
                        int64_t* d_makespan_ns, int32_t* d_status, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
   if (!d_demand || !h_model || !d_comm_ns || !d_makespan_ns || !d_status) return MOESCHED_EINVAL;
   if (!aligned4(d_demand) || !aligned4(d_status) || !aligned8(d_comm_ns) || !aligned8(d_makespan_ns))
     return MOESCHED_EINVAL;
   const moesched_model_t m = *h_model;
   if (!model_in_range(m)) return MOESCHED_EINVAL;
-  if (B == 0) return MOESCHED_OK;
   cudaError_t e = run_ideal_a2a(B, N, d_demand, m, reinterpret_cast<long long*>(d_comm_ns),
                                 reinterpret_cast<long long*>(d_makespan_ns), d_status,
                                 static_cast<cudaStream_t>(stream));

@@ -45,6 +45,7 @@ extern "C" int moesched_bvn_decompose_static(int B, int N, const int32_t* d_dema
                                              int32_t* d_coef, int32_t* d_count, int32_t* d_aug,
                                              int32_t* d_status, int64_t* d_work, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
   if (!d_demand || !d_perm || !d_coef || !d_count || !d_status) return MOESCHED_EINVAL;
   const uintptr_t misaligned = (reinterpret_cast<uintptr_t>(d_demand) | reinterpret_cast<uintptr_t>(d_coef) |
                                 reinterpret_cast<uintptr_t>(d_count) | reinterpret_cast<uintptr_t>(d_status) |
@@ -52,7 +53,6 @@ extern "C" int moesched_bvn_decompose_static(int B, int N, const int32_t* d_dema
   if (misaligned || (reinterpret_cast<uintptr_t>(d_work) & 7)) return MOESCHED_EINVAL;
   const size_t need = (size_t)B * N * bvn_scratch_stride(N);
   if (need > STATIC_SCRATCH_INTS) return MOESCHED_ETOOBIG;
-  if (B == 0) return MOESCHED_OK;
   int32_t* scratch = nullptr;
   cudaError_t e = scratch_address(&scratch);
   if (e == cudaSuccess)

@@ -190,3 +190,60 @@ def test_path_runner_matches_separate_calls(overlap):
         assert (path.score_mw[i] == sg[name]).all() and (path.score_bvn[i] == sv[name]).all()
     ref = oracle.schedule_eval(D, g.perm.cpu().numpy(), g.dur.cpu().numpy(), g.count.cpu().numpy(), DEFAULT_MODEL)
     assert (path.score_mw[0].cpu().numpy() == ref["makespan_overlap_ns"]).all()
+
+
+@pytest.mark.parametrize("N", [4, 8, 64, 128])
+def test_values_at_the_top_of_the_range(N):
+    """Entries up to 2^28 (greedy range) and sums up to 2^31-1 (BvN range): no 32-bit overflow."""
+    rng = np.random.default_rng(77 + N)
+    D = rng.integers(0, 2**28 + 1, size=(4, N, N)).astype(np.int32)
+    D[0, 0, 0] = 2**28                                   # exactly the greedy limit
+    D[1] = D[1] // (N * 2)                               # sums stay below 2^31: BvN accepts this one
+    D[2] = np.where(rng.random((N, N)) < 0.8, 0, D[2])   # sparse with huge entries
+    D[3, 1, 1] = 2**28 + 1                               # one above the limit: greedy rejects matrix 3
+    check_all(D, 12, 12)
+
+
+def test_empty_batch_is_a_no_op():
+    d = torch.zeros((0, 8, 8), dtype=torch.int32, device="cuda")
+    g = ms.mw_decompose(d, 4)
+    v = ms.bvn_decompose(d, 4)
+    s = ms.schedule_eval(d, g.perm, g.dur, g.count)
+    a = ms.ideal_a2a(d)
+    torch.cuda.synchronize()
+    assert g.count.numel() == 0 and v.count.numel() == 0 and s["status"].numel() == 0 and a["status"].numel() == 0
+
+
+def test_block_diagonal_and_staircase_matrices():
+    """Decomposable supports: several independent blocks, and a triangular staircase."""
+    N = 24
+    D = np.zeros((3, N, N), np.int32)
+    for k in range(0, N, 6):
+        D[0, k:k + 6, k:k + 6] = np.arange(1, 37).reshape(6, 6) + k
+    D[1] = np.triu(np.full((N, N), 5)) + np.eye(N, dtype=np.int32)
+    D[2] = np.tril(np.arange(N * N).reshape(N, N) % 7)
+    check_all(D, N * N, ms.bvn_capacity(N))
+
+
+def test_host_pipeline_returns_the_same_results_in_order():
+    batches = [make_demand(2, 64, seed=s) for s in (1, 2, 3, 4, 5)]
+    pipe = ms.HostPipeline(64, 16, 16)
+    slots = []
+    got = []
+    for i, D in enumerate(batches):
+        h = torch.from_numpy(D).pin_memory()
+        slots.append(pipe.submit(h))
+        if i >= 1:                                       # consume the previous batch while this one runs
+            got.append([t.clone() for t in pipe.result(slots[i - 1])])
+    got.append([t.clone() for t in pipe.result(slots[-1])])
+    for D, out in zip(batches, got):
+        ref = oracle.mw_decompose(D, 16, threads=4)
+        rv = oracle.bvn_decompose(D, ms.bvn_capacity(16), threads=4)
+        count, bcount = out[2].numpy(), out[6].numpy()
+        assert (count == ref["count"]).all() and (bcount == rv["count"]).all()
+        kk = np.arange(16)[None, :] < count[:, None]
+        assert (out[0].numpy()[kk] == ref["perm"][kk]).all() and (out[1].numpy()[kk] == ref["dur"][kk]).all()
+        kk = np.arange(rv["perm"].shape[1])[None, :] < bcount[:, None]
+        assert (out[4].numpy()[kk] == rv["perm"][kk]).all() and (out[5].numpy()[kk] == rv["coef"][kk]).all()
+        sc = oracle.schedule_eval(D, rv["perm"], rv["coef"], rv["count"], DEFAULT_MODEL)
+        assert (out[9].numpy()[0] == sc["makespan_overlap_ns"]).all()
