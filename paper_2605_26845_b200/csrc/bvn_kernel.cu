@@ -108,9 +108,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
                                                   long long* __restrict__ work_out) {
   constexpr int W = CPL;
   constexpr bool CLUSTER = MODE == 1;
-  // remembering which rows a search depended on pays off from N > 64 on (measured); below that the
-  // searches are so short that the bookkeeping costs more than the searches it saves
-  constexpr bool USE_MEMO = CPL >= 4;
+  constexpr bool USE_MEMO = true;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   WarpCtx cx;
   if constexpr (MODE == 2) cx = warp_prologue_global<CPL>(B, N, S, demand, scratch, smem_raw);

@@ -459,38 +459,83 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
 // row that already reached it before. changed = rows whose column changed since the last call.
 template <int W>
 struct CanonMemo {
+  // Up to 128 rows the per-row records live in registers: the lane keeps desc of rows
+  // lane, lane+32, ... (word k of a row set, bit `lane`), so collecting and recording are a
+  // few logic operations and one OR-reduction per word. Above that they live in shared memory.
+  static constexpr bool IN_REGS = W <= 4;
   unsigned known[W];
   unsigned changed[W];
+  unsigned dreg[IN_REGS ? W : 1][IN_REGS ? W : 1];
   __device__ __forceinline__ void reset() {
 #pragma unroll
     for (int w = 0; w < W; ++w) known[w] = changed[w] = 0u;
+    if constexpr (IN_REGS) {
+#pragma unroll
+      for (int k = 0; k < W; ++k)
+#pragma unroll
+        for (int w = 0; w < W; ++w) dreg[k][w] = 0u;
+    }
   }
 };
 
-// rows recorded as depending on any row of `rows`; their entries are consumed
+// rows recorded as depending on any row of `rows` are added to out; their entries are consumed
 template <int W>
 __device__ __forceinline__ void collect_dependants(int N, int lane, const unsigned (&rows)[W], unsigned* desc,
-                                                   unsigned (&out)[W]) {
-  unsigned left[W];
+                                                   CanonMemo<W>& memo, unsigned (&out)[W]) {
+  if constexpr (CanonMemo<W>::IN_REGS) {
+    unsigned acc[W];
 #pragma unroll
-  for (int w = 0; w < W; ++w) left[w] = rows[w];
-  for (int it = 0; it < N; ++it) {
-    const int r = lowest_bit<W>(left);
-    if (r < 0) break;
-    clear_bit<W>(left, r);
+    for (int w = 0; w < W; ++w) acc[w] = 0u;
 #pragma unroll
-    for (int w = 0; w < W; ++w) out[w] |= desc[r * W + w];
+    for (int k = 0; k < W; ++k) {
+      if ((rows[k] >> lane) & 1u) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) { acc[w] |= memo.dreg[k][w]; memo.dreg[k][w] = 0u; }
+      }
+    }
+#pragma unroll
+    for (int w = 0; w < W; ++w) out[w] |= __reduce_or_sync(FULL, acc[w]);
+  } else {
+    unsigned left[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) left[w] = rows[w];
+    for (int it = 0; it < N; ++it) {
+      const int r = lowest_bit<W>(left);
+      if (r < 0) break;
+      clear_bit<W>(left, r);
+#pragma unroll
+      for (int w = 0; w < W; ++w) out[w] |= desc[r * W + w];
+    }
+    __syncwarp();
+    // lane l clears the entries of the rows l, l+32, ... that were just read
+#pragma unroll
+    for (int k = 0; k < W; ++k) {
+      if ((rows[k] >> lane) & 1u) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) desc[(k * 32 + lane) * W + w] = 0u;
+      }
+    }
+    __syncwarp();
   }
-  __syncwarp();
-  // lane l clears the entries of the rows l, l+32, ... that were just read
+}
+
+// record that row i (one-hot imask) was searched and depends on the rows of anc
+template <int W>
+__device__ __forceinline__ void record_search(int lane, int i, const unsigned (&imask)[W], const unsigned (&anc)[W],
+                                              unsigned* desc, CanonMemo<W>& memo) {
 #pragma unroll
   for (int k = 0; k < W; ++k) {
-    if ((rows[k] >> lane) & 1u) {
+    if ((anc[k] >> lane) & 1u) {
+      if constexpr (CanonMemo<W>::IN_REGS) {
 #pragma unroll
-      for (int w = 0; w < W; ++w) desc[(k * 32 + lane) * W + w] = 0u;
+        for (int w = 0; w < W; ++w) memo.dreg[k][w] |= imask[w];
+      } else {
+        desc[(k * 32 + lane) * W + (i >> 5)] |= 1u << (i & 31);
+      }
     }
+    memo.known[k] |= imask[k];
   }
-  __syncwarp();
+  if constexpr (!CanonMemo<W>::IN_REGS) __syncwarp();
 }
 
 template <int CPL, bool MEMO>
@@ -505,7 +550,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
 #pragma unroll
   for (int w = 0; w < W; ++w) stale[w] = 0u;
   if constexpr (MEMO) {
-    collect_dependants<W>(N, lane, memo.changed, desc, stale);
+    collect_dependants<W>(N, lane, memo.changed, desc, memo, stale);
 #pragma unroll
     for (int w = 0; w < W; ++w) {
       stale[w] |= memo.changed[w];
@@ -578,15 +623,8 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
     const int sl = __shfl_sync(FULL, myslot, L);
     const int jstar = L * CPL + sl;
     if (jstar == xi) {
-      if constexpr (MEMO) {
-        // record: row i stays put until one of the rows that can reach it changes column
-#pragma unroll
-        for (int w = 0; w < W; ++w) {
-          if ((anc[w] >> lane) & 1u) desc[(w * 32 + lane) * W + (i >> 5)] |= 1u << (i & 31);
-          memo.known[w] |= imask[w];
-        }
-        __syncwarp();
-      }
+      // record: row i stays put until one of the rows that can reach it changes column
+      if constexpr (MEMO) record_search<W>(lane, i, imask, anc, desc, memo);
     } else {
       int cur = __shfl_sync(FULL, M.row_of(sl), L);   // row that gives up column jstar
       // level at which that row was reached
@@ -634,7 +672,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         unsigned hit[W];
 #pragma unroll
         for (int w = 0; w < W; ++w) hit[w] = moved[w];
-        collect_dependants<W>(N, lane, moved, desc, hit);
+        collect_dependants<W>(N, lane, moved, desc, memo, hit);
 #pragma unroll
         for (int w = 0; w < W; ++w) memo.known[w] &= ~hit[w];
       }
