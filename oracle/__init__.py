@@ -98,6 +98,24 @@ def schedule_eval(demand, perm, dur, count, model, threads=1):
     return out
 
 
+def schedule_prefix_eval(demand, perm, dur, count, model, threads=1):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    perm = np.ascontiguousarray(perm, dtype=np.uint8)
+    dur = np.ascontiguousarray(dur, dtype=np.int32)
+    count = np.ascontiguousarray(count, dtype=np.int32)
+    K = perm.shape[1]
+    m = np.array([int(model.get(f, 0)) for f in MODEL_FIELDS], np.int64)
+    po = np.zeros((B, K), np.int64)
+    pu = np.zeros((B, K), np.int64)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_schedule_prefix_eval(B, N, _p(d), K, _p(perm), _p(dur), _p(count), _p(m), _p(po), _p(pu),
+                                           _p(status), threads)
+    if rc != 0:
+        raise ValueError("oracle_schedule_prefix_eval rejected its arguments")
+    return dict(prefix_overlap_ns=po, prefix_unserved_tokens=pu, status=status)
+
+
 def ideal_a2a(demand, model):
     d = np.ascontiguousarray(demand, dtype=np.int32)
     B, N, _ = d.shape

@@ -524,6 +524,42 @@ int oracle_schedule_eval(int B, int N, const int32_t* demand, int k_stride, cons
   return 0;
 }
 
+// Scores of every prefix of a schedule: entry k is what oracle_schedule_eval returns for the first
+// k+1 matchings alone (the budget sweep of the greedy decomposition, Sec. 3.2 / 3.3: a smaller
+// budget is a prefix of the complete schedule). Written as exactly that: one evaluation per prefix.
+// Entries k >= count[b] are set to -1; a schedule that is bad as a whole gives status BAD_INPUT
+// and all entries -1.
+int oracle_schedule_prefix_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm,
+                                const int32_t* dur, const int32_t* count, const int64_t* model,
+                                int64_t* prefix_overlap_ns, int64_t* prefix_unserved_tokens,
+                                int32_t* status, int threads) {
+  if (B < 0 || N < 1 || N > 256 || k_stride < 1 || !demand || !perm || !dur || !count || !model) return -1;
+  Model m = {model[0], model[1], model[2], model[3], model[4], model[5]};
+  if (!model_ok(m)) return -1;
+  const size_t NN = (size_t)N * N;
+  parallel_for(B, threads, [&](int b) {
+    int64_t* po = prefix_overlap_ns + (size_t)b * k_stride;
+    int64_t* pu = prefix_unserved_tokens + (size_t)b * k_stride;
+    for (int k = 0; k < k_stride; ++k) po[k] = pu[k] = -1;
+    const int K = count[b];
+    status[b] = ST_BAD_INPUT;
+    if (K < 0 || K > k_stride) return;
+    i64 o, s, in, it, un;
+    int32_t st = ST_OK;
+    eval_one(N, demand + b * NN, K, perm + (size_t)b * k_stride * N, dur + (size_t)b * k_stride, m,
+             &o, &s, &in, &it, &un, &st);
+    if (st != ST_OK) return;
+    for (int k = 0; k < K; ++k) {
+      eval_one(N, demand + b * NN, k + 1, perm + (size_t)b * k_stride * N, dur + (size_t)b * k_stride, m,
+               &o, &s, &in, &it, &un, &st);
+      po[k] = o;
+      pu[k] = un;
+    }
+    status[b] = ST_OK;
+  });
+  return 0;
+}
+
 // Idealised congestion-free all-to-all [Sec. 4.1 "Comparisons": "the theoretical completion
 // time for a given communication matrix"]: every port sends and receives at line rate, so the
 // exchange lasts as long as the busiest port (largest row or column sum); like the sequential

@@ -221,3 +221,32 @@ def test_ideal_all_to_all_bound():
         assert g["dur"][b, :g["count"][b]].sum() >= port[b]
         link = sum(-(-int(c) * 14336 * 8 // 400) for c in v["coef"][b, :v["count"][b]])
         assert ideal["comm_ns"][b] <= link <= ideal["comm_ns"][b] + v["count"][b]
+
+
+def test_prefix_scores_are_the_scores_of_the_truncated_schedules():
+    """A smaller greedy budget yields a prefix (Sec. 3.2), so entry k of the prefix scores must be
+    the score of the decomposition run with budget k+1."""
+    D = make_demand(2, 5)
+    full = oracle.mw_decompose(D, 16)
+    pre = oracle.schedule_prefix_eval(D, full["perm"], full["dur"], full["count"], DEFAULT_MODEL)
+    for k in (1, 4, 9, 16):
+        part = oracle.mw_decompose(D, k)
+        sc = oracle.schedule_eval(D, part["perm"], part["dur"], part["count"], DEFAULT_MODEL)
+        assert (pre["prefix_overlap_ns"][:, k - 1] == sc["makespan_overlap_ns"]).all()
+        assert (pre["prefix_unserved_tokens"][:, k - 1] == sc["unserved_tokens"]).all()
+        assert (pre["prefix_unserved_tokens"][:, k - 1] == part["residual"].reshape(5, -1).sum(1)).all()
+    # makespan grows and unserved tokens shrink along the prefix
+    K = full["count"][0]
+    assert (np.diff(pre["prefix_overlap_ns"][0, :K]) > 0).all()
+    assert (np.diff(pre["prefix_unserved_tokens"][0, :K]) <= 0).all()
+    # hand case (same numbers as the three-matching example): combine ends 740, 785, 800
+    model = dict(bytes_per_token=50, link_gbps=40, reconfig_ns=5, expert_fixed_ns=100, expert_ps_per_token=1000)
+    D = np.array([[[30, 4], [2, 10]]], np.int32)
+    perm = np.array([[[0, 1], [1, 0], [0, 1], [0, 1]]], np.uint8)
+    dur = np.array([[30, 4, 1, 0]], np.int32)
+    pre = oracle.schedule_prefix_eval(D, perm, dur, np.array([3], np.int32), model)
+    assert list(pre["prefix_overlap_ns"][0]) == [740, 785, 800, -1]
+    assert list(pre["prefix_unserved_tokens"][0]) == [6, 0, 0, -1]
+    perm[0, 1] = [1, 1]
+    bad = oracle.schedule_prefix_eval(D, perm, dur, np.array([3], np.int32), model)
+    assert bad["status"][0] == -1 and (bad["prefix_overlap_ns"] == -1).all()
