@@ -196,6 +196,25 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride,
                            int32_t* d_status, void* stream);
 
 /*
+ * moesched_schedule_eval plus the scores of every prefix of the schedule (paper Sec. 3.3 asks how
+ * the ordering and number of matchings shape the makespan; a smaller greedy budget yields a prefix
+ * of the complete schedule, so one decomposition with the largest budget and this call give the
+ * whole budget sweep). For k < count[b]:
+ *   d_prefix_overlap_ns[b][k]      = makespan_overlap of matchings 0..k alone (= Cmb_{k+1})
+ *   d_prefix_unserved_tokens[b][k] = tokens of D not yet served after matchings 0..k
+ * Entries with k >= count[b], and all entries of a schedule flagged BAD_INPUT, are -1.
+ * Both arrays are [B][k_stride] int64 device memory; all other arguments as in
+ * moesched_schedule_eval.
+ */
+int moesched_schedule_prefix_eval(int B, int N, const int32_t* d_demand, int k_stride,
+                                  const uint8_t* d_perm, const int32_t* d_dur, const int32_t* d_count,
+                                  const moesched_model_t* h_model, int64_t* d_makespan_overlap_ns,
+                                  int64_t* d_makespan_serial_ns, int64_t* d_compute_idle_ns,
+                                  int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
+                                  int32_t* d_status, int64_t* d_prefix_overlap_ns,
+                                  int64_t* d_prefix_unserved_tokens, void* stream);
+
+/*
  * Idealised congestion-free all-to-all (paper Sec. 4.1 "Comparisons": "the theoretical
  * completion time for a given communication matrix"), the yardstick the decomposed
  * schedules are compared with. Every port sends and receives at line rate, so one exchange

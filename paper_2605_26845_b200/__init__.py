@@ -47,7 +47,8 @@ def load_library():
         lib = ctypes.CDLL(LIB_PATH)
         lib.moesched_strerror.restype = ctypes.c_char_p
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
-                     "moesched_schedule_eval", "moesched_ideal_a2a", "moesched_last_cuda_error"):
+                     "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
+                     "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         lib.moesched_probe_int_ops.restype = ctypes.c_longlong
@@ -223,10 +224,12 @@ SCORE_FIELDS = ("makespan_overlap_ns", "makespan_serial_ns", "compute_idle_ns", 
                 "unserved_tokens")
 
 
-def schedule_eval(demand, perm, dur, count, model=None, out=None, status=None) -> dict:
+def schedule_eval(demand, perm, dur, count, model=None, out=None, status=None, prefix=False) -> dict:
     """Score schedules under the dispatch-compute-combine model. Returns a dict of [B] int64
     tensors (SCORE_FIELDS) plus 'status' [B] int32; `out` may supply a [5, B] int64 tensor and
-    `status` a [B] int32 tensor."""
+    `status` a [B] int32 tensor. With prefix=True the dict also holds 'prefix_overlap_ns' and
+    'prefix_unserved_tokens', [B, k_stride] int64: the scores of the schedule cut after each
+    matching (-1 beyond count)."""
     lib = load_library()
     demand = _dev(demand, torch.int32, "demand")
     perm = _dev(perm, torch.uint8, "perm")
@@ -240,12 +243,19 @@ def schedule_eval(demand, perm, dur, count, model=None, out=None, status=None) -
     scores = out if out is not None else torch.empty((5, B), dtype=torch.int64, device=dev)
     if status is None:
         status = torch.empty(B, dtype=torch.int32, device=dev)
+    K = int(perm.shape[1])
+    pre = torch.empty((2, B, K), dtype=torch.int64, device=dev) if prefix else None
     with torch.cuda.device(dev):
-        rc = lib.moesched_schedule_eval(B, N, _ptr(demand), int(perm.shape[1]), _ptr(perm), _ptr(dur), _ptr(count),
-                                        ctypes.byref(m), _ptr(scores[0]), _ptr(scores[1]), _ptr(scores[2]),
-                                        _ptr(scores[3]), _ptr(scores[4]), _ptr(status), _stream(dev))
+        args = (B, N, _ptr(demand), K, _ptr(perm), _ptr(dur), _ptr(count), ctypes.byref(m), _ptr(scores[0]),
+                _ptr(scores[1]), _ptr(scores[2]), _ptr(scores[3]), _ptr(scores[4]), _ptr(status))
+        if prefix:
+            rc = lib.moesched_schedule_prefix_eval(*args, _ptr(pre[0]), _ptr(pre[1]), _stream(dev))
+        else:
+            rc = lib.moesched_schedule_eval(*args, _stream(dev))
     _check(rc, "moesched_schedule_eval")
     res = {name: scores[i] for i, name in enumerate(SCORE_FIELDS)}
+    if prefix:
+        res["prefix_overlap_ns"], res["prefix_unserved_tokens"] = pre[0], pre[1]
     res["status"] = status
     return res
 

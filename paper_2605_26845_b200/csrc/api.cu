@@ -81,11 +81,12 @@ int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uin
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }
 
-int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
-                           const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
-                           int64_t* d_makespan_overlap_ns, int64_t* d_makespan_serial_ns,
-                           int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
-                           int32_t* d_status, void* stream) {
+static int schedule_eval_impl(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                              const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                              int64_t* d_makespan_overlap_ns, int64_t* d_makespan_serial_ns,
+                              int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
+                              int32_t* d_status, int64_t* d_prefix_overlap_ns, int64_t* d_prefix_unserved_tokens,
+                              void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_stride < 1) return MOESCHED_EINVAL;
   if (B == 0) return MOESCHED_OK;
   if (!d_demand || !d_perm || !d_dur || !d_count || !h_model || !d_makespan_overlap_ns ||
@@ -93,7 +94,8 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
     return MOESCHED_EINVAL;
   if (!aligned4(d_demand) || !aligned4(d_dur) || !aligned4(d_count) || !aligned4(d_status) ||
       !aligned8(d_makespan_overlap_ns) || !aligned8(d_makespan_serial_ns) || !aligned8(d_compute_idle_ns) ||
-      !aligned8(d_link_idle_tokens) || !aligned8(d_unserved_tokens))
+      !aligned8(d_link_idle_tokens) || !aligned8(d_unserved_tokens) || !aligned8(d_prefix_overlap_ns) ||
+      !aligned8(d_prefix_unserved_tokens))
     return MOESCHED_EINVAL;
   const moesched_model_t m = *h_model;
   if (!model_in_range(m)) return MOESCHED_EINVAL;
@@ -103,8 +105,32 @@ int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, 
                            reinterpret_cast<long long*>(d_compute_idle_ns),
                            reinterpret_cast<long long*>(d_link_idle_tokens),
                            reinterpret_cast<long long*>(d_unserved_tokens), d_status,
+                           reinterpret_cast<long long*>(d_prefix_overlap_ns),
+                           reinterpret_cast<long long*>(d_prefix_unserved_tokens),
                            static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_schedule_eval(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                           const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                           int64_t* d_makespan_overlap_ns, int64_t* d_makespan_serial_ns,
+                           int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens, int64_t* d_unserved_tokens,
+                           int32_t* d_status, void* stream) {
+  return schedule_eval_impl(B, N, d_demand, k_stride, d_perm, d_dur, d_count, h_model, d_makespan_overlap_ns,
+                            d_makespan_serial_ns, d_compute_idle_ns, d_link_idle_tokens, d_unserved_tokens,
+                            d_status, nullptr, nullptr, stream);
+}
+
+int moesched_schedule_prefix_eval(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                                  const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                                  int64_t* d_makespan_overlap_ns, int64_t* d_makespan_serial_ns,
+                                  int64_t* d_compute_idle_ns, int64_t* d_link_idle_tokens,
+                                  int64_t* d_unserved_tokens, int32_t* d_status, int64_t* d_prefix_overlap_ns,
+                                  int64_t* d_prefix_unserved_tokens, void* stream) {
+  if (B > 0 && (!d_prefix_overlap_ns || !d_prefix_unserved_tokens)) return MOESCHED_EINVAL;
+  return schedule_eval_impl(B, N, d_demand, k_stride, d_perm, d_dur, d_count, h_model, d_makespan_overlap_ns,
+                            d_makespan_serial_ns, d_compute_idle_ns, d_link_idle_tokens, d_unserved_tokens,
+                            d_status, d_prefix_overlap_ns, d_prefix_unserved_tokens, stream);
 }
 
 int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_model_t* h_model, int64_t* d_comm_ns,

@@ -708,7 +708,7 @@ inline int bvn_scratch_stride(int N) { return (N + 7) / 8 * 8; }
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
-                     cudaStream_t stream);
+                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream);
 
 bool model_in_range(const moesched_model_t& m);
 cudaError_t run_ideal_a2a(int B, int N, const int32_t* demand, const moesched_model_t& model, long long* comm_ns,

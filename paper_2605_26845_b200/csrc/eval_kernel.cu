@@ -57,13 +57,17 @@ __device__ __forceinline__ Packed<CPL> load_dest(const uint8_t* row, int lane, i
   return p;
 }
 
-template <int CPL, bool CLUSTER>
+// PREFIX: also write, after every matching k, the overlap makespan and the unserved tokens of the
+// schedule cut after k+1 matchings (entries beyond count, or all entries of a bad schedule, are -1).
+template <int CPL, bool CLUSTER, bool PREFIX>
 __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_stride,
                                                    const uint8_t* __restrict__ perm, const int32_t* __restrict__ dur,
                                                    const int32_t* __restrict__ count, moesched_model_t model,
                                                    long long* __restrict__ overlap, long long* __restrict__ serial,
                                                    long long* __restrict__ idle_ns, long long* __restrict__ idle_tok,
-                                                   long long* __restrict__ unserved, int32_t* __restrict__ status) {
+                                                   long long* __restrict__ unserved, int32_t* __restrict__ status,
+                                                   long long* __restrict__ prefix_overlap,
+                                                   long long* __restrict__ prefix_unserved) {
   constexpr int W = CPL;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
@@ -79,7 +83,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   const int K = count[b];
   if (K < 0 || K > k_stride) bad = 1;
 
-  long long dsp = 0, cmp = 0, cmb = 0, ser = 0, comp_sum = 0, dsp1 = 0, dur_sum = 0;
+  long long dsp = 0, cmp = 0, cmb = 0, ser = 0, comp_sum = 0, dsp1 = 0, dur_sum = 0, served_sum = 0;
   const uint8_t* pb = perm + (size_t)b * k_stride * N;
   const int32_t* db = dur + (size_t)b * k_stride;
 
@@ -111,6 +115,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
 #pragma unroll
           for (int w = 0; w < W; ++w) cols[w] = 0u;
           int g = 0, oob = 0;
+          unsigned slo = 0u, shi = 0u;   // served tokens of this matching, low and high halves
 #pragma unroll
           for (int s = 0; s < CPL; ++s) {
             const int r = lane * CPL + s;
@@ -123,6 +128,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
                 const int sv = min(dk, val);
                 *p = val - sv;
                 g = max(g, sv);
+                if constexpr (PREFIX) { slo += (unsigned)sv & 0xffffu; shi += (unsigned)sv >> 16; }
               } else {
                 oob = 1;
               }
@@ -144,6 +150,13 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
             ser += 2 * leg + comp;
             comp_sum += comp;
             dur_sum += dk;
+            if constexpr (PREFIX) {
+              served_sum += ((long long)__reduce_add_sync(FULL, shi) << 16) + __reduce_add_sync(FULL, slo);
+              if (lane == 0) {
+                prefix_overlap[(size_t)b * k_stride + k0 + q] = cmb;
+                prefix_unserved[(size_t)b * k_stride + k0 + q] = total - served_sum;
+              }
+            }
           }
           __syncwarp();
         }
@@ -156,6 +169,13 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   if (!bad) {
     __syncwarp();
     left = matrix_sum<CPL>(D, N, lane, lane_in, nullptr);
+  }
+  if constexpr (PREFIX) {
+    const int from = bad ? 0 : K;
+    for (int k = from + lane; k < k_stride; k += 32) {
+      prefix_overlap[(size_t)b * k_stride + k] = -1;
+      prefix_unserved[(size_t)b * k_stride + k] = -1;
+    }
   }
   if (lane == 0) {
     if (bad) {
@@ -176,11 +196,19 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
-                     cudaStream_t stream) {
+                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream) {
   const Geometry ge = plan_geometry(N);
-#define MOESCHED_GO(C, CL)                                                                                       \
-  return launch_warp_kernel(eval_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, count, \
-                            model, overlap, serial, idle_ns, idle_tok, unserved, status)
+  const bool prefix = prefix_overlap != nullptr;
+#define MOESCHED_GO(C, CL)                                                                                        \
+  do {                                                                                                            \
+    if (prefix)                                                                                                   \
+      return launch_warp_kernel(eval_kernel<C, CL, true>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, \
+                                count, model, overlap, serial, idle_ns, idle_tok, unserved, status,              \
+                                prefix_overlap, prefix_unserved);                                                 \
+    return launch_warp_kernel(eval_kernel<C, CL, false>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur,  \
+                              count, model, overlap, serial, idle_ns, idle_tok, unserved, status,                \
+                              prefix_overlap, prefix_unserved);                                                   \
+  } while (0)
   if (ge.cluster) MOESCHED_GO(8, true);
   switch (ge.cpl) {
     case 1: MOESCHED_GO(1, false);

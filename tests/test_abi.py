@@ -26,7 +26,7 @@ def declared_functions():
 
 def test_header_declares_the_entry_points():
     names = declared_functions()
-    for want in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval", "moesched_ideal_a2a",
+    for want in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_schedule_eval", "moesched_ideal_a2a", "moesched_schedule_prefix_eval",
                  "moesched_strerror", "moesched_last_cuda_error"):
         assert want in names
 

@@ -193,3 +193,26 @@ def test_ideal_all_to_all_at_full_size(cfg):
     total = torch.where(used(s), s.dur, torch.zeros_like(s.dur)).sum(1).to(torch.int64)
     port = torch.maximum(d.sum(1).max(1).values, d.sum(2).max(1).values)
     assert (total[complete] >= port[complete]).all()
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 5])
+def test_budget_sweep_from_one_decomposition(cfg):
+    """The greedy schedule with the largest budget plus its prefix scores reproduce the scores of
+    every smaller budget of the configuration."""
+    D, d = demand(cfg)
+    B = D.shape[0]
+    budgets = CONFIGS[cfg]["k_max"]
+    full = ms.mw_decompose(d, max(budgets))
+    pre = ms.schedule_eval(d, full.perm, full.dur, full.count, DEFAULT_MODEL, prefix=True)
+    rows = sample_rows(B, 16)
+    rnp = rows.cpu().numpy()
+    for k in budgets:
+        part = ms.mw_decompose(d, k)
+        sc = ms.schedule_eval(d, part.perm, part.dur, part.count, DEFAULT_MODEL)
+        last = (part.count - 1).clamp(min=0).to(torch.int64)[:, None]
+        some = part.count > 0
+        assert (pre["prefix_overlap_ns"].gather(1, last)[:, 0][some] == sc["makespan_overlap_ns"][some]).all()
+        assert (pre["prefix_unserved_tokens"].gather(1, last)[:, 0][some] == sc["unserved_tokens"][some]).all()
+        ref = oracle.mw_decompose(D[rnp], k, threads=THREADS)
+        osc = oracle.schedule_eval(D[rnp], ref["perm"], ref["dur"], ref["count"], DEFAULT_MODEL, threads=THREADS)
+        assert (sc["makespan_overlap_ns"][rows].cpu().numpy() == osc["makespan_overlap_ns"]).all()

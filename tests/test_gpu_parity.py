@@ -247,3 +247,30 @@ def test_host_pipeline_returns_the_same_results_in_order():
         assert (out[4].numpy()[kk] == rv["perm"][kk]).all() and (out[5].numpy()[kk] == rv["coef"][kk]).all()
         sc = oracle.schedule_eval(D, rv["perm"], rv["coef"], rv["count"], DEFAULT_MODEL)
         assert (out[9].numpy()[0] == sc["makespan_overlap_ns"]).all()
+
+
+@pytest.mark.parametrize("N", [3, 16, 33, 64, 128, 256])
+def test_prefix_scores(N):
+    D = random_matrices(5, N, seed=6000 + N, kind="uniform", high=500, zero_frac=0.4)
+    d = dev(D)
+    k = min(12, N * N)
+    for sched, key in ((ms.mw_decompose(d, k), "dur"), (ms.bvn_decompose(d, k), "coef")):
+        perm = sched.perm.cpu().numpy().copy()
+        dur = sched.dur.cpu().numpy().copy()
+        count = sched.count.cpu().numpy().copy()
+        kk = np.arange(k)[None, :] < count[:, None]
+        perm[~kk] = 0
+        dur[~kk] = 0
+        perm[4, 0, 0] = perm[4, 0, N - 1] if N > 1 else 200          # matrix 4: a bad schedule
+        if N == 1:
+            perm[4, 0, 0] = 200
+        if count[4] == 0:
+            count[4] = 1
+        got = ms.schedule_eval(d, dev(perm), dev(dur), dev(count), DEFAULT_MODEL, prefix=True)
+        ref = oracle.schedule_prefix_eval(D, perm, dur, count, DEFAULT_MODEL, threads=4)
+        plain = oracle.schedule_eval(D, perm, dur, count, DEFAULT_MODEL, threads=4)
+        assert (got["status"].cpu().numpy() == ref["status"]).all() and ref["status"][4] == -1
+        for name in ("prefix_overlap_ns", "prefix_unserved_tokens"):
+            assert (got[name].cpu().numpy() == ref[name]).all(), name
+        for name in ms.SCORE_FIELDS:
+            assert (got[name].cpu().numpy() == plain[name]).all(), name
