@@ -208,6 +208,33 @@ __device__ __forceinline__ RowVec<CPL> load_cols(const int* rowp, int lane) {
   return r;
 }
 
+// The same matrix held as 16-bit entries (all values <= 65535): half the shared memory per
+// matrix, hence twice the matrices per SM for the kernels that shared memory limits.
+struct MatView16 {
+  unsigned short* base;
+  int S;   // row stride in entries, a multiple of CPL
+  __device__ __forceinline__ unsigned short* row(int r) const { return base + r * S; }
+};
+
+template <int CPL>
+__device__ __forceinline__ RowVec<CPL> load_cols(const unsigned short* rowp, int lane) {
+  RowVec<CPL> r;
+  if constexpr (CPL == 1) {
+    r.v[0] = rowp[lane];
+  } else if constexpr (CPL == 2) {
+    const unsigned t = *reinterpret_cast<const unsigned*>(rowp + lane * 2);
+    r.v[0] = t & 0xffffu; r.v[1] = t >> 16;
+  } else if constexpr (CPL == 4) {
+    const uint2 t = *reinterpret_cast<const uint2*>(rowp + lane * 4);
+    r.v[0] = t.x & 0xffffu; r.v[1] = t.x >> 16; r.v[2] = t.y & 0xffffu; r.v[3] = t.y >> 16;
+  } else {
+    const uint4 t = *reinterpret_cast<const uint4*>(rowp + lane * 8);
+    r.v[0] = t.x & 0xffffu; r.v[1] = t.x >> 16; r.v[2] = t.y & 0xffffu; r.v[3] = t.y >> 16;
+    r.v[4] = t.z & 0xffffu; r.v[5] = t.z >> 16; r.v[6] = t.w & 0xffffu; r.v[7] = t.w >> 16;
+  }
+  return r;
+}
+
 // ---- bulk asynchronous copy global -> shared with an mbarrier ---------------------------
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) {
@@ -382,6 +409,45 @@ __device__ __forceinline__ WarpCtx warp_prologue_global(int B, int N, int S, con
   const int32_t* src = demand + (size_t)cx.b * N * N;
   for (int r = 0; r < N; ++r)
     for (int c = cx.lane; c < S; c += 32) mat[(size_t)r * S + c] = c < N ? src[(size_t)r * N + c] : 0;
+  __syncwarp();
+  return cx;
+}
+
+// Variant for matrices whose entries all fit 16 bits: the warp's shared memory is
+// [N x S entries of 16 bits][hist][x]; the entries are narrowed while they are loaded.
+__host__ __device__ inline size_t warp_smem_bytes16(int N, int S, int W) {
+  return align16((size_t)N * S * 2) + hist_bytes_for(N, W) + align16((size_t)N * 2);
+}
+
+struct WarpCtx16 {
+  int b;
+  int lane;
+  MatView16 M;
+  unsigned* hist;
+  short* x;
+  bool worker;
+};
+
+template <int CPL>
+__device__ __forceinline__ WarpCtx16 warp_prologue16(int B, int N, int S, const int32_t* demand,
+                                                     unsigned char* smem_raw) {
+  WarpCtx16 cx;
+  cx.lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int wpb = blockDim.x >> 5;
+  unsigned char* base = smem_raw + (size_t)warp * warp_smem_bytes16(N, S, CPL);
+  const size_t mat_bytes = align16((size_t)N * S * 2);
+  cx.M.base = reinterpret_cast<unsigned short*>(base);
+  cx.M.S = S;
+  cx.hist = reinterpret_cast<unsigned*>(base + mat_bytes);
+  cx.x = reinterpret_cast<short*>(base + mat_bytes + hist_bytes_for(N, CPL));
+  cx.b = blockIdx.x * wpb + warp;
+  cx.worker = cx.b < B;
+  if (!cx.worker) return cx;
+  const int32_t* src = demand + (size_t)cx.b * N * N;
+  for (int r = 0; r < N; ++r)
+    for (int c = cx.lane; c < S; c += 32)
+      cx.M.base[r * S + c] = c < N ? (unsigned short)src[(size_t)r * N + c] : (unsigned short)0;
   __syncwarp();
   return cx;
 }

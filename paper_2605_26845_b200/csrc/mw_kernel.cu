@@ -6,6 +6,8 @@
 // the row duals, marks the tight edges and hands that graph to canonicalise(),
 // which returns the lexicographically smallest optimal permutation. The matched
 // entries are then served whole; the largest one is the matching's duration.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace moesched {
@@ -23,8 +25,8 @@ struct MwState {
 // it if that column is still free: such a row is matched along a tight edge. The rows left
 // over are added one by one by a shortest-augmenting-path search that settles one column
 // per scan and updates only the column duals. Returns false if an iteration limit was hit.
-template <int CPL>
-__device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int lane, bool lane_in,
+template <int CPL, typename View>
+__device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane, bool lane_in,
                                                  MwState<CPL>& st, short* x, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
   constexpr int W = CPL;
   bool ok = true;
@@ -137,20 +139,52 @@ __device__ __forceinline__ bool solve_assignment(const MatView& R, int N, int la
   return ok;
 }
 
-template <int CPL, bool CLUSTER>
+// Matrices are sorted into two classes by a streaming pre-pass that leaves the class in status[b]:
+// all entries within 16 bits (held as 16-bit values: twice as many matrices per SM) or not.
+constexpr int CLASS_U16 = 64;
+constexpr int CLASS_I32 = 65;
+
+__global__ void __launch_bounds__(256) mw_classify_kernel(int B, int N, const int32_t* __restrict__ demand,
+                                                          int32_t* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (b >= B) return;
+  const int32_t* D = demand + (size_t)b * N * N;
+  int wide = 0;
+  for (int e = lane; e < N * N; e += 32) wide |= (unsigned)D[e] > 65535u;   // negative entries count as wide
+  wide = __any_sync(FULL, wide);
+  if (lane == 0) status[b] = wide ? CLASS_I32 : CLASS_U16;
+}
+
+// MODE 0: matrix in this CTA's shared memory as int32; 1: split over a 2-CTA cluster; 2: 16-bit entries.
+// only_class != 0: handle only the matrices whose status[b] holds that class.
+template <int CPL, int MODE>
 __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                  uint8_t* __restrict__ perm, int32_t* __restrict__ dur,
                                                  int32_t* __restrict__ count, int32_t* __restrict__ residual,
-                                                 int32_t* __restrict__ status, long long* __restrict__ work_out) {
+                                                 int32_t* status, long long* __restrict__ work_out, int only_class) {
   constexpr int W = CPL;
+  constexpr bool CLUSTER = MODE == 1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
-  if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
-  const int lane = cx.lane, b = cx.b;
-  const MatView R = cx.M;
-  short* x = cx.x;
-  unsigned* hist = cx.hist;
-  const bool loaded = cx.loaded;
+  if (only_class != 0) {
+    const int bb = CLUSTER ? (int)(blockIdx.x >> 1) : (int)(blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
+    if (bb < B && status[bb] != only_class) return;   // both CTAs of a cluster see the same class
+  }
+  using View = typename std::conditional<MODE == 2, MatView16, MatView>::type;
+  View R;
+  int lane, b;
+  short* x;
+  unsigned* hist;
+  bool loaded = true;
+  if constexpr (MODE == 2) {
+    WarpCtx16 cx = warp_prologue16<CPL>(B, N, S, demand, smem_raw);
+    if (!cx.worker) return;
+    lane = cx.lane; b = cx.b; R = cx.M; x = cx.x; hist = cx.hist;
+  } else {
+    WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+    if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
+    lane = cx.lane; b = cx.b; R = cx.M; x = cx.x; hist = cx.hist; loaded = cx.loaded;
+  }
 
   unsigned work[MOESCHED_WORK_FIELDS];
 #pragma unroll
@@ -192,7 +226,7 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
     uint8_t* pout = perm + (size_t)b * k_max * N;
     int32_t* dout = dur + (size_t)b * k_max;
     while (k < k_max && nnz > 0) {
-      if (!solve_assignment<CPL>(R, N, lane, lane_in, st, x, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
+      if (!solve_assignment<CPL, View>(R, N, lane, lane_in, st, x, work)) { st_code = MOESCHED_ST_INTERNAL; break; }
       // tight edges: row r is tight to column c iff cost(r,c) - v[c] equals the row minimum
       unsigned C[CPL][CPL];
 #pragma unroll
@@ -230,7 +264,7 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
       for (int s = 0; s < CPL; ++s) {
         const int c = lane * CPL + s;
         if (c < N && st.M.mr[s] >= 0) {
-          int* p = R.row(st.M.mr[s]) + c;
+          auto* p = R.row(st.M.mr[s]) + c;
           const int val = *p;
           dmax = max(dmax, val);
           served += val != 0;
@@ -256,7 +290,7 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
   if (residual != nullptr && st_code != MOESCHED_ST_BAD_INPUT) {
     int32_t* ro = residual + (size_t)b * N * N;
     for (int r = 0; r < N; ++r) {
-      const int* rp = R.row(r);
+      const auto* rp = R.row(r);
       for (int c = lane; c < N; c += 32) ro[(size_t)r * N + c] = rp[c];
     }
   }
@@ -269,20 +303,43 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
 
 // ---- host side ---------------------------------------------------------------------------
 
+template <int MODE>
+static cudaError_t launch_mw_mode(Geometry ge, int B, int N, const int32_t* demand, int k_max, uint8_t* perm,
+                                  int32_t* dur, int32_t* count, int32_t* residual, int32_t* status, long long* work,
+                                  int only_class, cudaStream_t stream) {
+#define MOESCHED_GO(C)                                                                                      \
+  return launch_warp_kernel(mw_kernel<C, MODE>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur, count, \
+                            residual, status, work, only_class)
+  switch (ge.cpl) {
+    case 1: MOESCHED_GO(1);
+    case 2: MOESCHED_GO(2);
+    case 4: MOESCHED_GO(4);
+    default: MOESCHED_GO(8);
+  }
+#undef MOESCHED_GO
+}
+
 cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
                    int32_t* residual, int32_t* status, long long* work, cudaStream_t stream) {
   const Geometry ge = plan_geometry(N);
-#define MOESCHED_GO(C, CL)                                                                                  \
-  return launch_warp_kernel(mw_kernel<C, CL>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur, count, \
-                            residual, status, work)
-  if (ge.cluster) MOESCHED_GO(8, true);
-  switch (ge.cpl) {
-    case 1: MOESCHED_GO(1, false);
-    case 2: MOESCHED_GO(2, false);
-    case 4: MOESCHED_GO(4, false);
-    default: MOESCHED_GO(8, false);
+  int only_class = 0;
+  if (N >= 48) {
+    // Shared memory limits how many matrices an SM holds: first the matrices that fit 16-bit entries
+    // (one CTA each at any N), then the rest as int32 (a 2-CTA cluster above N = 232).
+    mw_classify_kernel<<<(B + 7) / 8, 256, 0, stream>>>(B, N, demand, status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    Geometry g16 = ge;
+    g16.cluster = false;
+    g16.wpb = 1;
+    g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
+    e = launch_mw_mode<2>(g16, B, N, demand, k_max, perm, dur, count, residual, status, work, CLASS_U16, stream);
+    if (e != cudaSuccess) return e;
+    only_class = CLASS_I32;
   }
-#undef MOESCHED_GO
+  if (ge.cluster) return launch_mw_mode<1>(ge, B, N, demand, k_max, perm, dur, count, residual, status, work,
+                                           only_class, stream);
+  return launch_mw_mode<0>(ge, B, N, demand, k_max, perm, dur, count, residual, status, work, only_class, stream);
 }
 
 }  // namespace moesched

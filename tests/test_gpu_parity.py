@@ -274,3 +274,15 @@ def test_prefix_scores(N):
             assert (got[name].cpu().numpy() == ref[name]).all(), name
         for name in ms.SCORE_FIELDS:
             assert (got[name].cpu().numpy() == plain[name]).all(), name
+
+
+@pytest.mark.parametrize("N", [48, 64, 100, 200, 256])
+def test_mixed_16_bit_and_wide_matrices_in_one_batch(N):
+    """The greedy path holds matrices whose entries fit 16 bits in a narrower layout; a batch may mix both."""
+    D = random_matrices(6, N, seed=7000 + N, kind="uniform", high=60000, zero_frac=0.3)
+    D[1] *= 3                                          # entries up to 180000: wide
+    D[2, 5 % N, 7 % N] = 65535                         # the largest narrow value
+    D[3, 5 % N, 7 % N] = 65536                         # the smallest wide value
+    D[4] = 0
+    D[5, 0, 0] = -2                                    # bad input goes through the wide path
+    check_all(D, 5, 5)
