@@ -776,6 +776,11 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                      long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream);
 
+// class codes the pre-pass leaves in status[b] (never equal to a final status)
+constexpr int CLASS_U16 = 64;
+constexpr int CLASS_I32 = 65;
+cudaError_t classify_matrices(int B, int N, const int32_t* demand, int32_t* status, cudaStream_t stream);
+
 bool model_in_range(const moesched_model_t& m);
 cudaError_t run_ideal_a2a(int B, int N, const int32_t* demand, const moesched_model_t& model, long long* comm_ns,
                           long long* makespan_ns, int32_t* status, cudaStream_t stream);

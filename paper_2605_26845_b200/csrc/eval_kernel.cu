@@ -18,8 +18,8 @@ __device__ __forceinline__ long long warp_sum64(long long v) {
   return v;
 }
 
-template <int CPL>
-__device__ __forceinline__ long long matrix_sum(const MatView& M, int N, int lane, bool lane_in, int* any_negative) {
+template <int CPL, typename View>
+__device__ __forceinline__ long long matrix_sum(const View& M, int N, int lane, bool lane_in, int* any_negative) {
   long long acc = 0;
   int neg = 0;
   for (int r = 0; r < N; ++r) {
@@ -59,26 +59,42 @@ __device__ __forceinline__ Packed<CPL> load_dest(const uint8_t* row, int lane, i
 
 // PREFIX: also write, after every matching k, the overlap makespan and the unserved tokens of the
 // schedule cut after k+1 matchings (entries beyond count, or all entries of a bad schedule, are -1).
-template <int CPL, bool CLUSTER, bool PREFIX>
+// MODE 0: demand in this CTA's shared memory as int32; 1: split over a 2-CTA cluster; 2: held as
+// 16-bit entries (matrices the pre-pass classified as narrow). only_class as in the greedy kernel.
+template <int CPL, int MODE, bool PREFIX>
 __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_stride,
                                                    const uint8_t* __restrict__ perm, const int32_t* __restrict__ dur,
                                                    const int32_t* __restrict__ count, moesched_model_t model,
                                                    long long* __restrict__ overlap, long long* __restrict__ serial,
                                                    long long* __restrict__ idle_ns, long long* __restrict__ idle_tok,
-                                                   long long* __restrict__ unserved, int32_t* __restrict__ status,
+                                                   long long* __restrict__ unserved, int32_t* status,
                                                    long long* __restrict__ prefix_overlap,
-                                                   long long* __restrict__ prefix_unserved) {
+                                                   long long* __restrict__ prefix_unserved, int only_class) {
   constexpr int W = CPL;
+  constexpr bool CLUSTER = MODE == 1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
-  if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
-  const int lane = cx.lane, b = cx.b;
-  const MatView D = cx.M;
+  if (only_class != 0) {
+    const int bb = CLUSTER ? (int)(blockIdx.x >> 1) : (int)(blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
+    if (bb < B && status[bb] != only_class) return;
+  }
+  using View = typename std::conditional<MODE == 2, MatView16, MatView>::type;
+  View D;
+  int lane, b;
+  bool loaded = true;
+  if constexpr (MODE == 2) {
+    WarpCtx16 cx = warp_prologue16<CPL>(B, N, S, demand, smem_raw);
+    if (!cx.worker) return;
+    lane = cx.lane; b = cx.b; D = cx.M;
+  } else {
+    WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
+    if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
+    lane = cx.lane; b = cx.b; D = cx.M; loaded = cx.loaded;
+  }
   const bool lane_in = lane * CPL < S;
 
-  int bad = cx.loaded ? 0 : 1;
+  int bad = loaded ? 0 : 1;
   int neg = 0;
-  const long long total = matrix_sum<CPL>(D, N, lane, lane_in, &neg);
+  const long long total = matrix_sum<CPL, View>(D, N, lane, lane_in, &neg);
   bad |= neg;
   const int K = count[b];
   if (K < 0 || K > k_stride) bad = 1;
@@ -123,7 +139,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
               const int j = (int)((dest[q].v >> (8 * s)) & 0xff);
               if (j < N) {
                 set_bit<W>(cols, j);
-                int* p = D.row(r) + j;
+                auto* p = D.row(r) + j;
                 const int val = *p;
                 const int sv = min(dk, val);
                 *p = val - sv;
@@ -168,7 +184,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   long long left = 0;
   if (!bad) {
     __syncwarp();
-    left = matrix_sum<CPL>(D, N, lane, lane_in, nullptr);
+    left = matrix_sum<CPL, View>(D, N, lane, lane_in, nullptr);
   }
   if constexpr (PREFIX) {
     const int from = bad ? 0 : K;
@@ -193,30 +209,57 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   cluster_epilogue<CLUSTER>();
 }
 
+template <int MODE>
+static cudaError_t launch_eval_mode(const Geometry& ge, int B, int N, const int32_t* demand, int k_stride,
+                                    const uint8_t* perm, const int32_t* dur, const int32_t* count,
+                                    const moesched_model_t& model, long long* overlap, long long* serial,
+                                    long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
+                                    long long* prefix_overlap, long long* prefix_unserved, int only_class,
+                                    cudaStream_t stream) {
+  const bool prefix = prefix_overlap != nullptr;
+#define MOESCHED_GO(C)                                                                                             \
+  do {                                                                                                             \
+    if (prefix)                                                                                                    \
+      return launch_warp_kernel(eval_kernel<C, MODE, true>, ge, B, stream, B, N, ge.S, demand, k_stride, perm,     \
+                                dur, count, model, overlap, serial, idle_ns, idle_tok, unserved, status,          \
+                                prefix_overlap, prefix_unserved, only_class);                                      \
+    return launch_warp_kernel(eval_kernel<C, MODE, false>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, \
+                              count, model, overlap, serial, idle_ns, idle_tok, unserved, status, prefix_overlap, \
+                              prefix_unserved, only_class);                                                        \
+  } while (0)
+  switch (ge.cpl) {
+    case 1: MOESCHED_GO(1);
+    case 2: MOESCHED_GO(2);
+    case 4: MOESCHED_GO(4);
+    default: MOESCHED_GO(8);
+  }
+#undef MOESCHED_GO
+}
+
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                      long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream) {
   const Geometry ge = plan_geometry(N);
-  const bool prefix = prefix_overlap != nullptr;
-#define MOESCHED_GO(C, CL)                                                                                        \
-  do {                                                                                                            \
-    if (prefix)                                                                                                   \
-      return launch_warp_kernel(eval_kernel<C, CL, true>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, \
-                                count, model, overlap, serial, idle_ns, idle_tok, unserved, status,              \
-                                prefix_overlap, prefix_unserved);                                                 \
-    return launch_warp_kernel(eval_kernel<C, CL, false>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur,  \
-                              count, model, overlap, serial, idle_ns, idle_tok, unserved, status,                \
-                              prefix_overlap, prefix_unserved);                                                   \
-  } while (0)
-  if (ge.cluster) MOESCHED_GO(8, true);
-  switch (ge.cpl) {
-    case 1: MOESCHED_GO(1, false);
-    case 2: MOESCHED_GO(2, false);
-    case 4: MOESCHED_GO(4, false);
-    default: MOESCHED_GO(8, false);
+  int only_class = 0;
+  if (N >= 48) {
+    // as in the greedy path: narrow matrices first, in the 16-bit layout, then the rest
+    cudaError_t e = classify_matrices(B, N, demand, status, stream);
+    if (e != cudaSuccess) return e;
+    Geometry g16 = ge;
+    g16.cluster = false;
+    g16.wpb = 1;
+    g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
+    e = launch_eval_mode<2>(g16, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok,
+                            unserved, status, prefix_overlap, prefix_unserved, CLASS_U16, stream);
+    if (e != cudaSuccess) return e;
+    only_class = CLASS_I32;
   }
-#undef MOESCHED_GO
+  if (ge.cluster)
+    return launch_eval_mode<1>(ge, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns,
+                               idle_tok, unserved, status, prefix_overlap, prefix_unserved, only_class, stream);
+  return launch_eval_mode<0>(ge, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok,
+                             unserved, status, prefix_overlap, prefix_unserved, only_class, stream);
 }
 
 }  // namespace moesched

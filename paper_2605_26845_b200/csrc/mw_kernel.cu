@@ -141,9 +141,6 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
 
 // Matrices are sorted into two classes by a streaming pre-pass that leaves the class in status[b]:
 // all entries within 16 bits (held as 16-bit values: twice as many matrices per SM) or not.
-constexpr int CLASS_U16 = 64;
-constexpr int CLASS_I32 = 65;
-
 __global__ void __launch_bounds__(256) mw_classify_kernel(int B, int N, const int32_t* __restrict__ demand,
                                                           int32_t* __restrict__ status) {
   const int lane = threadIdx.x & 31;
@@ -301,6 +298,11 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
   cluster_epilogue<CLUSTER>();
 }
 
+cudaError_t classify_matrices(int B, int N, const int32_t* demand, int32_t* status, cudaStream_t stream) {
+  mw_classify_kernel<<<(B + 7) / 8, 256, 0, stream>>>(B, N, demand, status);
+  return cudaGetLastError();
+}
+
 // ---- host side ---------------------------------------------------------------------------
 
 template <int MODE>
@@ -326,8 +328,7 @@ cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm
   if (N >= 48) {
     // Shared memory limits how many matrices an SM holds: first the matrices that fit 16-bit entries
     // (one CTA each at any N), then the rest as int32 (a 2-CTA cluster above N = 232).
-    mw_classify_kernel<<<(B + 7) / 8, 256, 0, stream>>>(B, N, demand, status);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = classify_matrices(B, N, demand, status, stream);
     if (e != cudaSuccess) return e;
     Geometry g16 = ge;
     g16.cluster = false;
