@@ -26,6 +26,18 @@ Geometry plan_geometry(int N) {
   return ge;
 }
 
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 static int fail_cuda(cudaError_t e) {
   g_last_cuda_error = (int)e;
   return MOESCHED_ECUDA;

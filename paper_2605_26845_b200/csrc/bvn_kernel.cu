@@ -315,7 +315,9 @@ cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* per
     // working copy in global memory: four matrices per CTA, shared memory only for hist and x
     ge.cluster = false;
     ge.S = bvn_scratch_stride(N);
-    ge.wpb = 4;
+    // four matrices per CTA once there are enough of them to give every SM several CTAs;
+    // a small batch is spread one matrix per CTA so that no SM sits idle
+    ge.wpb = B >= 16 * sm_count() ? 4 : 1;
     ge.smem = warp_smem_bytes_global(N, ge.cpl) * ge.wpb;
     switch (ge.cpl) {
       case 1: MOESCHED_GO(1, 2);

@@ -764,6 +764,7 @@ struct Geometry {
   size_t smem;   // dynamic shared memory per CTA
 };
 Geometry plan_geometry(int N);
+int sm_count();   // SMs of the current device (148 on B200), cached per device
 
 cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
                    int32_t* residual, int32_t* status, long long* work, cudaStream_t stream);
