@@ -29,13 +29,14 @@ import numpy as np  # noqa: E402
 from paper_2605_26845_b200.workload import CONFIGS, DEFAULT_MODEL, SEED, bvn_capacity, make_demand  # noqa: E402
 
 METRIC = "demand-matrix decompositions/sec at N=64 (greedy+BvN)"
+UNIT = "decompositions/s"
+CFG = 3        # the headline workload; --config selects another of the five
+K_MW = 64      # greedy budget = the largest k_max of the configuration
+FALLBACK_HBM_GBS = 6650.0
 
 
 def metric_name():
     return METRIC.replace("N=64", f"N={CONFIGS[CFG]['N']}")
-UNIT = "decompositions/s"
-CFG = 3        # the headline workload; --config selects another of the five
-K_MW = 64      # greedy budget = the largest k_max of the configuration
 
 
 def select_config(cfg):
@@ -43,7 +44,7 @@ def select_config(cfg):
     CFG = cfg
     K_MW = max(CONFIGS[cfg]["k_max"])
 
-FALLBACK_HBM_GBS = 6650.0
+
 # Issue-rate ceiling for plain integer work: 148 SMs x 4 warp schedulers x 32 lanes, one
 # instruction per scheduler per clock, at the SM clock sampled during the run.
 ALU_LANES_PER_CLK = 148 * 4 * 32

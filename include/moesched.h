@@ -30,6 +30,9 @@
  *     for a null pointer or an out-of-range size (nothing enqueued); B = 0 is
  *     accepted, enqueues nothing and does not look at the pointers;
  *     MOESCHED_ECUDA when a CUDA call failed (moesched_last_cuda_error()).
+ *   - d_status doubles as working memory while a call runs (from N = 48 up the greedy and
+ *     scoring entry points park a per-matrix class code there between their kernels); it
+ *     holds the outcome once the stream has passed the call.
  *   - Per-matrix outcome in d_status[b]:
  *       MOESCHED_ST_OK          complete result
  *       MOESCHED_ST_TRUNCATED   k_max matchings written, matrix not exhausted
