@@ -122,11 +122,13 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
         dest[q].v = 0;
         if (q < kend && lane * CPL < N) dest[q] = load_dest<CPL>(pb + (size_t)(k0 + q) * N, lane, N, packed_ok);
       }
+      // replay: lane q keeps what matching k0+q served (largest pair, total)
+      int g_mine = 0;
+      long long served_mine = 0;
 #pragma unroll
       for (int q = 0; q < 32; ++q) {
         if (q < kend && !bad) {
           const int dk = __shfl_sync(FULL, dk_mine, q);
-          const long long t = __shfl_sync(FULL, t_mine, q);
           unsigned cols[W];
 #pragma unroll
           for (int w = 0; w < W; ++w) cols[w] = 0u;
@@ -157,25 +159,45 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
             bad = 1;
           } else {
             g = __reduce_max_sync(FULL, g);
-            const long long comp = batch_time_ns(model, g);
-            const long long leg = model.reconfig_ns + t;
-            dsp += leg;
-            if (k0 + q == 0) dsp1 = dsp;
-            cmp = max(dsp, cmp) + comp;
-            cmb = max(cmp, cmb) + leg;
-            ser += 2 * leg + comp;
-            comp_sum += comp;
-            dur_sum += dk;
+            if (lane == q) g_mine = g;
             if constexpr (PREFIX) {
-              served_sum += ((long long)__reduce_add_sync(FULL, shi) << 16) + __reduce_add_sync(FULL, slo);
-              if (lane == 0) {
-                prefix_overlap[(size_t)b * k_stride + k0 + q] = cmb;
-                prefix_unserved[(size_t)b * k_stride + k0 + q] = total - served_sum;
-              }
+              const long long sv_all = ((long long)__reduce_add_sync(FULL, shi) << 16) + __reduce_add_sync(FULL, slo);
+              if (lane == q) served_mine = sv_all;
             }
           }
           __syncwarp();
         }
+      }
+      if (bad) break;
+      // times of the chunk, one matching per lane, then the three-stage recurrence in order
+      const bool mine = lane < kend;
+      const long long comp_mine = mine ? batch_time_ns(model, g_mine) : 0;
+      const long long leg_mine = mine ? model.reconfig_ns + t_mine : 0;
+      ser += warp_sum64(2 * leg_mine + comp_mine);
+      comp_sum += warp_sum64(comp_mine);
+      dur_sum += warp_sum64((long long)dk_mine);
+      long long cmb_mine = 0;
+      for (int q = 0; q < kend; ++q) {
+        const long long leg = __shfl_sync(FULL, leg_mine, q);
+        const long long comp = __shfl_sync(FULL, comp_mine, q);
+        dsp += leg;
+        if (k0 + q == 0) dsp1 = dsp;
+        cmp = max(dsp, cmp) + comp;
+        cmb = max(cmp, cmb) + leg;
+        if (PREFIX && lane == q) cmb_mine = cmb;
+      }
+      if constexpr (PREFIX) {
+        long long run = served_mine;   // inclusive prefix sum over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const long long up = __shfl_up_sync(FULL, run, o);
+          if (lane >= o) run += up;
+        }
+        if (mine) {
+          prefix_overlap[(size_t)b * k_stride + k0 + lane] = cmb_mine;
+          prefix_unserved[(size_t)b * k_stride + k0 + lane] = total - (served_sum + run);
+        }
+        served_sum += __shfl_sync(FULL, run, 31);
       }
     }
     if (dur_sum > (1LL << 40)) bad = 1;
