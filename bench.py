@@ -215,6 +215,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="matrices per GPU (default: the configuration's B)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the step from a CUDA graph (pays off when the kernels take microseconds)")
     ap.add_argument("--overlap", action="store_true",
                     help="fork greedy and BvN onto two streams (measured slower than one stream)")
     ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS),
@@ -263,7 +265,10 @@ def main():
         if events is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-        path.run(d, DEFAULT_MODEL, overlap=args.overlap)
+        if args.graph:
+            path.run_graph(d, DEFAULT_MODEL)
+        else:
+            path.run(d, DEFAULT_MODEL, overlap=args.overlap)
         if events is not None:
             e1.record(stream)
             events.append((e0, e1))
@@ -374,6 +379,7 @@ def main():
             "config": {"workload": workload_name(B), "l2": "flushed between timed steps (256 MiB write, untimed)",
                        "matchings_per_matrix": {"greedy": k_mw, "bvn": k_bv}, "all_status_ok": ok,
                        "streams": "greedy and BvN forked on two streams, joined" if args.overlap else "one",
+                       "launch": "CUDA graph replay" if args.graph else "direct",
                        "seed": SEED},
             "kernels_ms": {n: float(t) for n, t in zip(names, per_kernel)},
             "kernels_ms_note": "per-kernel events from a second, identical serial pass",
@@ -393,7 +399,9 @@ def main():
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "how": "HostPipeline: upload, kernels and download on three streams, two slots",
                     "results_match_device_run": e2e_ok},
-            "gpu_launches": 4 * args.steps,
+            # per step: greedy, BvN and two scoring launches; from N = 48 up the greedy and scoring entry
+            # points each add a class pre-pass and a second (wide-class) launch
+            "gpu_launches": (4 if N < 48 else 10) * args.steps,
             "clocks": ck,
         }
         if world == 1 and not args.no_cpu_baseline:

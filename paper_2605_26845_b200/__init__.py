@@ -305,6 +305,21 @@ class Path:
         schedule_eval(demand, self.bvn.perm, self.bvn.dur, self.bvn.count, model, out=self.score_bvn,
                       status=self.eval_status_bvn)
 
+    def run_graph(self, demand, model=None):
+        """The same launches replayed from a CUDA graph: for small matrices the step is a handful of
+        microsecond kernels and the cost of launching them one by one dominates. The graph is captured
+        on first use and again whenever the demand tensor's address or the model changes."""
+        key = (demand.data_ptr(), tuple(sorted((model or DEFAULT_MODEL).items())))
+        if getattr(self, "_graph_key", None) != key:
+            self.run(demand, model)                      # first-use set-up outside the capture
+            torch.cuda.current_stream(self.device).synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                self.run(demand, model)
+            self._graph, self._graph_key, self._graph_demand = graph, key, demand
+        self._graph.replay()
+        return self
+
     def run(self, demand, model=None, overlap=False):
         """Enqueue the four kernels; results are ready when the caller's current stream reaches this point."""
         if not overlap:

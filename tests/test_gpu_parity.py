@@ -286,3 +286,19 @@ def test_mixed_16_bit_and_wide_matrices_in_one_batch(N):
     D[4] = 0
     D[5, 0, 0] = -2                                    # bad input goes through the wide path
     check_all(D, 5, 5)
+
+
+def test_graph_replay_gives_the_same_schedules():
+    D = make_demand(1, 64)
+    d = dev(D)
+    path = ms.Path(64, 8, 8)
+    for _ in range(3):
+        path.run_graph(d, DEFAULT_MODEL)
+    d2 = dev(make_demand(1, 64, seed=5))                 # another tensor: the graph is captured again
+    other = ms.Path(64, 8, 8).run(d2)
+    path.run_graph(d2, DEFAULT_MODEL)
+    torch.cuda.synchronize()
+    for a, b in ((path.mw, other.mw), (path.bvn, other.bvn)):
+        kk = torch.arange(a.perm.shape[1], device="cuda")[None, :] < b.count[:, None]
+        assert (a.count == b.count).all() and (a.perm[kk] == b.perm[kk]).all() and (a.dur[kk] == b.dur[kk]).all()
+    assert (path.score_bvn == other.score_bvn).all() and (path.score_mw == other.score_mw).all()
