@@ -12,6 +12,29 @@
 
 namespace moesched {
 
+// Division by a divisor fixed for the whole launch (the link speed): floor(x / d) for
+// 0 <= x < 2^55 as a multiply-high and a shift (Granlund-Montgomery: with l = ceil(log2 d) and
+// m = ceil(2^(55+l) / d), m*d lies in [2^(55+l), 2^(55+l) + 2^l], which makes the quotient exact
+// for every 55-bit x).
+struct FastDiv {
+  unsigned long long m;
+  int sh;
+};
+static FastDiv make_fastdiv(long long d) {
+  int l = 0;
+  while ((1LL << l) < d) ++l;
+  const unsigned __int128 num = (unsigned __int128)1 << (55 + l);
+  FastDiv f;
+  f.m = (unsigned long long)((num + (unsigned __int128)(d - 1)) / (unsigned __int128)d);
+  f.sh = 55 + l;
+  return f;
+}
+__device__ __forceinline__ long long fast_div(long long x, const FastDiv& f) {
+  const unsigned long long hi = __umul64hi(f.m, (unsigned long long)x);
+  const unsigned long long lo = f.m * (unsigned long long)x;
+  return (long long)(f.sh >= 64 ? hi >> (f.sh - 64) : (hi << (64 - f.sh)) | (lo >> f.sh));
+}
+
 __device__ __forceinline__ long long warp_sum64(long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
@@ -65,7 +88,7 @@ template <int CPL, int MODE, bool PREFIX>
 __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_stride,
                                                    const uint8_t* __restrict__ perm, const int32_t* __restrict__ dur,
                                                    const int32_t* __restrict__ count, moesched_model_t model,
-                                                   long long* __restrict__ overlap, long long* __restrict__ serial,
+                                                   FastDiv by_gbps, long long* __restrict__ overlap, long long* __restrict__ serial,
                                                    long long* __restrict__ idle_ns, long long* __restrict__ idle_tok,
                                                    long long* __restrict__ unserved, int32_t* status,
                                                    long long* __restrict__ prefix_overlap,
@@ -111,8 +134,9 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
       const int kk = k0 + lane;
       const int dk_mine = kk < K ? db[kk] : 0;
       if (__any_sync(FULL, dk_mine < 0)) { bad = 1; break; }
+      // dk < 2^31, bytes_per_token and link_gbps <= 2^20: the dividend stays below 2^55
       const long long t_mine =
-          ((long long)dk_mine * model.bytes_per_token * 8 + model.link_gbps - 1) / model.link_gbps;
+          fast_div((long long)dk_mine * model.bytes_per_token * 8 + model.link_gbps - 1, by_gbps);
       const int kend = min(32, K - k0);
       // fetch the lane's destinations of all matchings of the chunk before using any of them:
       // 32 independent loads in flight instead of one dependent load per matching
@@ -239,15 +263,16 @@ static cudaError_t launch_eval_mode(const Geometry& ge, int B, int N, const int3
                                     long long* prefix_overlap, long long* prefix_unserved, int only_class,
                                     cudaStream_t stream) {
   const bool prefix = prefix_overlap != nullptr;
+  const FastDiv by_gbps = make_fastdiv(model.link_gbps);
 #define MOESCHED_GO(C)                                                                                             \
   do {                                                                                                             \
     if (prefix)                                                                                                    \
       return launch_warp_kernel(eval_kernel<C, MODE, true>, ge, B, stream, B, N, ge.S, demand, k_stride, perm,     \
-                                dur, count, model, overlap, serial, idle_ns, idle_tok, unserved, status,          \
-                                prefix_overlap, prefix_unserved, only_class);                                      \
+                                dur, count, model, by_gbps, overlap, serial, idle_ns, idle_tok, unserved,         \
+                                status, prefix_overlap, prefix_unserved, only_class);                              \
     return launch_warp_kernel(eval_kernel<C, MODE, false>, ge, B, stream, B, N, ge.S, demand, k_stride, perm, dur, \
-                              count, model, overlap, serial, idle_ns, idle_tok, unserved, status, prefix_overlap, \
-                              prefix_unserved, only_class);                                                        \
+                              count, model, by_gbps, overlap, serial, idle_ns, idle_tok, unserved, status,        \
+                              prefix_overlap, prefix_unserved, only_class);                                        \
   } while (0)
   switch (ge.cpl) {
     case 1: MOESCHED_GO(1);

@@ -111,6 +111,30 @@ def test_eval_rejects_bad_schedules():
         assert (s[name].cpu().numpy() == r[name]).all(), name
 
 
+@pytest.mark.parametrize("gbps", [1, 2, 3, 7, 400, 1000, 4099, 65536, 2**20 - 1, 2**20])
+def test_link_time_for_any_link_speed_and_token_size(gbps):
+    """The kernel divides by the link speed with a multiply-high by a constant made on the host; the
+    quotient must equal the plain ceiling division of the definition for every speed and size in range."""
+    N = 5
+    rng = np.random.default_rng(gbps)
+    durs = np.array([1, 2, 3, 25, 2**31 - 1, 2**30 + 1, 999_983, 2**20, 2**20 + 1, 123_456_789], dtype=np.int32)
+    K = len(durs)
+    B = 4
+    D = rng.integers(0, 2**31 - 1, size=(B, N, N), dtype=np.int64).astype(np.int32)
+    perm = np.stack([np.stack([rng.permutation(N) for _ in range(K)]) for _ in range(B)]).astype(np.uint8)
+    dur = np.stack([rng.permutation(durs) for _ in range(B)]).astype(np.int32)
+    count = np.full(B, K, dtype=np.int32)
+    for nbytes in (1, 50, 14336, 2**20 - 1, 2**20):
+        model = dict(DEFAULT_MODEL, link_gbps=gbps, bytes_per_token=nbytes)
+        s = ms.schedule_eval(dev(D), dev(perm), dev(dur), dev(count), model, prefix=True)
+        r = oracle.schedule_eval(D, perm, dur, count, model)
+        assert (r["status"] == 0).all()
+        for name in ms.SCORE_FIELDS + ("status",):
+            assert (s[name].cpu().numpy() == r[name]).all(), (name, nbytes)
+        rp = oracle.schedule_prefix_eval(D, perm, dur, count, model)
+        assert (s["prefix_overlap_ns"].cpu().numpy() == rp["prefix_overlap_ns"]).all()
+
+
 def test_argument_errors_are_reported():
     d = dev(make_demand(1, 2))
     with pytest.raises(ms.MoeschedError):
