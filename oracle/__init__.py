@@ -22,7 +22,7 @@ MODEL_FIELDS = ("bytes_per_token", "link_gbps", "reconfig_ns", "expert_fixed_ns"
 def build(force: bool = False) -> str:
     """Compile the oracle with g++ (no CUDA involved)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        cmd = ["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _SO, _SRC]
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-shared", "-fPIC", "-pthread", "-o", _SO, _SRC]
         subprocess.run(cmd, check=True)
     return _SO
 
@@ -126,6 +126,32 @@ def ideal_a2a(demand, model):
     if lib().oracle_ideal_a2a(B, N, _p(d), _p(m), _p(comm), _p(mk), _p(status)) != 0:
         raise ValueError("oracle_ideal_a2a rejected its arguments")
     return dict(comm_ns=comm, makespan_ns=mk, status=status)
+
+
+def sinkhorn_scale(demand, iters, smooth, scale_bits, threads=1):
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    scaled = np.zeros((B, N, N), np.float64)
+    fixed = np.zeros((B, N, N), np.int32)
+    stretch = np.zeros(B, np.float64)
+    row_err = np.zeros(B, np.float64)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_sinkhorn_scale(B, N, _p(d), int(iters), ctypes.c_double(smooth), int(scale_bits), _p(scaled),
+                                     _p(fixed), _p(stretch), _p(row_err), _p(status), threads)
+    if rc != 0:
+        raise ValueError("oracle_sinkhorn_scale rejected its arguments")
+    return dict(scaled=scaled, fixed=fixed, stretch=stretch, row_err=row_err, status=status)
+
+
+def sinkhorn_durations(coef, count, stretch, scale_bits):
+    coef = np.ascontiguousarray(coef, dtype=np.int32)
+    count = np.ascontiguousarray(count, dtype=np.int32)
+    stretch = np.ascontiguousarray(stretch, dtype=np.float64)
+    B, K = coef.shape
+    dur = np.zeros((B, K), np.int32)
+    if lib().oracle_sinkhorn_durations(B, K, _p(coef), _p(count), _p(stretch), int(scale_bits), _p(dur)) != 0:
+        raise ValueError("oracle_sinkhorn_durations rejected its arguments")
+    return dur
 
 
 def max_weight_perm(W, tier):

@@ -43,6 +43,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <limits>
@@ -587,6 +588,98 @@ int oracle_ideal_a2a(int B, int N, const int32_t* demand, const int64_t* model, 
     comm_ns[b] = t;
     makespan_ns[b] = 2 * t + batch_time(m, recv);
     status[b] = ST_OK;
+  }
+  return 0;
+}
+
+// Sinkhorn-Knopp scaling [Sec. 3.1: the preprocessing the paper names for making a demand matrix
+// doubly stochastic before the Birkhoff-von Neumann decomposition]. The paper gives no constants,
+// so the steps are spelled out here: X = D + smooth (smooth > 0 gives every pair a little mass, so
+// that zero rows and columns can be scaled at all); one sweep divides every row by its sum, then
+// every column by its sum; `iters` sweeps. All arithmetic is IEEE double, sums run left to right
+// (rows) and top to bottom (columns), one rounding per operation.
+//   scaled   = the matrix after the last sweep (column sums 1 up to rounding, row sums 1 + row_err);
+//   fixed    = round-half-up(scaled * 2^scale_bits): the integer matrix handed to the exact
+//              Birkhoff decomposition (its padding absorbs the rounding residue);
+//   stretch  = max over pairs with demand of D_ij * 2^scale_bits / fixed_ij: how many tokens one
+//              unit of the scaled schedule must carry so that every pair with a positive fixed
+//              entry can send all its demand -- pairs scaled up by the balancing finish early and
+//              idle, which is the bubble the paper describes;
+//   status   = BAD_INPUT (negative entry, or a row or column without mass), TRUNCATED (a pair with
+//              demand was rounded to zero and cannot be served), else OK.
+int oracle_sinkhorn_scale(int B, int N, const int32_t* demand, int iters, double smooth, int scale_bits,
+                          double* scaled, int32_t* fixed, double* stretch, double* row_err, int32_t* status,
+                          int threads) {
+  if (B < 0 || N < 1 || N > 256 || iters < 1 || !(smooth >= 0.0) || scale_bits < 1 || scale_bits > 24 ||
+      !demand || !scaled || !fixed || !stretch || !row_err || !status)
+    return -1;
+  const double scale = (double)(1 << scale_bits);
+  parallel_for(B, threads, [&](int b) {
+    const int32_t* D = demand + (size_t)b * N * N;
+    double* S = scaled + (size_t)b * N * N;
+    int32_t* Q = fixed + (size_t)b * N * N;
+    bool bad = false;
+    for (int e = 0; e < N * N; ++e) {
+      if (D[e] < 0) bad = true;
+      S[e] = (double)D[e] + smooth;
+    }
+    for (int it = 0; it < iters && !bad; ++it) {
+      for (int i = 0; i < N; ++i) {
+        double r = 0.0;
+        for (int j = 0; j < N; ++j) r = r + S[i * N + j];
+        if (!(r > 0.0)) bad = true;
+        for (int j = 0; j < N; ++j) S[i * N + j] = S[i * N + j] / r;
+      }
+      for (int j = 0; j < N; ++j) {
+        double c = 0.0;
+        for (int i = 0; i < N; ++i) c = c + S[i * N + j];
+        if (!(c > 0.0)) bad = true;
+        for (int i = 0; i < N; ++i) S[i * N + j] = S[i * N + j] / c;
+      }
+    }
+    if (bad) {
+      for (int e = 0; e < N * N; ++e) { S[e] = 0.0; Q[e] = 0; }
+      stretch[b] = 0.0;
+      row_err[b] = 0.0;
+      status[b] = ST_BAD_INPUT;
+      return;
+    }
+    double err = 0.0, st = 0.0;
+    bool dropped = false;
+    for (int i = 0; i < N; ++i) {
+      double r = 0.0;
+      for (int j = 0; j < N; ++j) r = r + S[i * N + j];
+      const double d = r - 1.0;
+      err = std::max(err, d < 0.0 ? -d : d);
+    }
+    for (int e = 0; e < N * N; ++e) {
+      const double q = std::floor(S[e] * scale + 0.5);
+      Q[e] = (int32_t)q;
+      if (D[e] > 0) {
+        if (Q[e] > 0) st = std::max(st, ((double)D[e] * scale) / (double)Q[e]);
+        else dropped = true;
+      }
+    }
+    stretch[b] = st;
+    row_err[b] = err;
+    status[b] = dropped ? ST_TRUNCATED : ST_OK;
+  });
+  return 0;
+}
+
+// Length in tokens of each matching of a decomposition of `fixed`: coefficient c (in units of
+// 2^-scale_bits of the scaled schedule) times the matrix's stretch, rounded up; capped at 2^31-1.
+int oracle_sinkhorn_durations(int B, int k_stride, const int32_t* coef, const int32_t* count,
+                              const double* stretch, int scale_bits, int32_t* dur) {
+  if (B < 0 || k_stride < 1 || scale_bits < 1 || scale_bits > 24 || !coef || !count || !stretch || !dur) return -1;
+  const double scale = (double)(1 << scale_bits);
+  for (int b = 0; b < B; ++b) {
+    const int K = std::min(std::max(count[b], 0), k_stride);
+    for (int k = 0; k < K; ++k) {
+      const double x = (double)coef[(size_t)b * k_stride + k] * stretch[b];
+      const double d = std::ceil(x / scale);
+      dur[(size_t)b * k_stride + k] = d >= 2147483647.0 ? I32_MAX : (d > 0.0 ? (int32_t)d : 0);
+    }
   }
   return 0;
 }
