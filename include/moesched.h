@@ -237,6 +237,54 @@ int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_mod
                        int64_t* d_comm_ns, int64_t* d_makespan_ns, int32_t* d_status, void* stream);
 
 /*
+ * Sinkhorn-Knopp scaling: the preprocessing the paper names for the Birkhoff-von Neumann
+ * decomposition (Sec. 3.1: "a preprocessing step such as Sinkhorn-Knopp normalization is
+ * required before decomposition can be applied"; it "redistributes communication mass across
+ * rows and columns" and so "introduces idle capacity that does not correspond to the original
+ * routing demand"). moesched_bvn_decompose pads instead; this entry point gives the paper's
+ * multiplicative route: scale here, then decompose d_fixed with moesched_bvn_decompose, turn
+ * its coefficients into token counts with moesched_sinkhorn_durations, and score the result
+ * against the ORIGINAL demand with moesched_schedule_eval.
+ *
+ * The paper fixes no constants; the steps are: X = D + smooth; one sweep divides every row of X
+ * by its sum and then every column by its sum; `iters` sweeps. IEEE double arithmetic, row sums
+ * accumulated left to right and column sums top to bottom, one rounding per operation -- the
+ * result is therefore reproducible bit for bit.
+ *   d_scaled[b]  = X after the last sweep (column sums 1 up to rounding)
+ *   d_row_err[b] = max_i |sum_j scaled[b][i][j] - 1|, the distance from double stochasticity
+ *   d_fixed[b]   = floor(scaled * 2^scale_bits + 0.5), the integer matrix for the exact
+ *                  decomposition (its padding absorbs the rounding residue)
+ *   d_stretch[b] = max over pairs with D_ij > 0 and fixed_ij > 0 of D_ij * 2^scale_bits / fixed_ij:
+ *                  tokens per unit of the scaled schedule such that every such pair can send all of
+ *                  its demand; pairs that the balancing scaled up finish early and idle
+ *   d_status[b]  = OK; TRUNCATED when a pair with demand was rounded to zero (it cannot be served);
+ *                  BAD_INPUT for a negative entry or a row or column without mass (possible only
+ *                  with smooth = 0): all outputs of that matrix are then 0.
+ *
+ *   d_demand   in   [B][N][N] int32, entries >= 0
+ *   iters      in   number of sweeps, >= 1
+ *   smooth     in   >= 0, added to every entry (gives empty rows and columns mass)
+ *   scale_bits in   1..24
+ *   d_scaled   out  [B][N][N] double, 8-byte aligned; also the working memory of the call
+ *   d_fixed    out  [B][N][N] int32
+ *   d_stretch, d_row_err  out  [B] double;  d_status  out  [B] int32
+ */
+int moesched_sinkhorn_scale(int B, int N, const int32_t* d_demand, int iters, double smooth, int scale_bits,
+                            double* d_scaled, int32_t* d_fixed, double* d_stretch, double* d_row_err,
+                            int32_t* d_status, void* stream);
+
+/*
+ * Length in tokens of every matching of a decomposition of d_fixed (paper Sec. 3.1: a matching
+ * with coefficient lambda occupies that share of the scaled schedule):
+ *   d_dur[b][k] = min(2^31-1, ceil(d_coef[b][k] * d_stretch[b] / 2^scale_bits))  for k < d_count[b],
+ * in double arithmetic (one rounding in the product; the division by a power of two is exact).
+ * Entries with k >= d_count[b] are left untouched. All arrays are device memory:
+ * d_coef, d_dur [B][k_stride] int32, d_count [B] int32, d_stretch [B] double.
+ */
+int moesched_sinkhorn_durations(int B, int k_stride, const int32_t* d_coef, const int32_t* d_count,
+                                const double* d_stretch, int scale_bits, int32_t* d_dur, void* stream);
+
+/*
  * Birkhoff-von Neumann decomposition for callers that cannot allocate device memory.
  * (The paper has no counterpart: this is a packaging variant of moesched_bvn_decompose,
  * same arguments, same results, minus d_scratch.)

@@ -48,7 +48,7 @@ def load_library():
         lib.moesched_strerror.restype = ctypes.c_char_p
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
                      "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
-                     "moesched_last_cuda_error"):
+                     "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         lib.moesched_probe_int_ops.restype = ctypes.c_longlong
@@ -197,6 +197,41 @@ def probe_int_rate(device=None, blocks=148 * 8, iters=20000, reps=3) -> float:
             e1.synchronize()
             best = max(best, ops / (e0.elapsed_time(e1) * 1e-3))
     return best
+
+
+def sinkhorn_scale(demand, iters=20, smooth=0.5, scale_bits=20) -> dict:
+    """Sinkhorn-Knopp scaling of a batch (paper Sec. 3.1). Returns scaled [B, N, N] float64, fixed
+    [B, N, N] int32 (= round(scaled * 2^scale_bits), the input of bvn_decompose), stretch [B], row_err [B]
+    float64 and status [B]."""
+    demand = _check_demand(demand)
+    B, N, _ = demand.shape
+    dev = demand.device
+    out = dict(scaled=torch.empty((B, N, N), dtype=torch.float64, device=dev),
+               fixed=torch.empty((B, N, N), dtype=torch.int32, device=dev),
+               stretch=torch.empty(B, dtype=torch.float64, device=dev),
+               row_err=torch.empty(B, dtype=torch.float64, device=dev),
+               status=torch.empty(B, dtype=torch.int32, device=dev))
+    rc = load_library().moesched_sinkhorn_scale(B, N, _ptr(demand), int(iters), ctypes.c_double(float(smooth)),
+                                                int(scale_bits), _ptr(out["scaled"]), _ptr(out["fixed"]),
+                                                _ptr(out["stretch"]), _ptr(out["row_err"]), _ptr(out["status"]),
+                                                _stream(dev))
+    _check(rc, "moesched_sinkhorn_scale")
+    return out
+
+
+def sinkhorn_durations(coef, count, stretch, scale_bits=20, out=None) -> torch.Tensor:
+    """Token length of each matching of a decomposition of sinkhorn_scale(...)["fixed"]:
+    ceil(coef * stretch / 2^scale_bits) for the first count[b] matchings of every schedule."""
+    coef = _dev(coef, torch.int32, "coef")
+    count = _dev(count, torch.int32, "count")
+    stretch = _dev(stretch, torch.float64, "stretch")
+    B, K = coef.shape
+    if out is None:
+        out = torch.zeros_like(coef)
+    rc = load_library().moesched_sinkhorn_durations(B, K, _ptr(coef), _ptr(count), _ptr(stretch), int(scale_bits),
+                                                    _ptr(_dev(out, torch.int32, "out")), _stream(coef.device))
+    _check(rc, "moesched_sinkhorn_durations")
+    return out
 
 
 def _model(model):

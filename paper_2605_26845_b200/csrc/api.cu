@@ -160,6 +160,32 @@ int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_mod
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }
 
+int moesched_sinkhorn_scale(int B, int N, const int32_t* d_demand, int iters, double smooth, int scale_bits,
+                            double* d_scaled, int32_t* d_fixed, double* d_stretch, double* d_row_err,
+                            int32_t* d_status, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || iters < 1 || !(smooth >= 0.0) || scale_bits < 1 || scale_bits > 24)
+    return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_demand || !d_scaled || !d_fixed || !d_stretch || !d_row_err || !d_status) return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_fixed) || !aligned4(d_status) || !aligned8(d_scaled) ||
+      !aligned8(d_stretch) || !aligned8(d_row_err))
+    return MOESCHED_EINVAL;
+  cudaError_t e = run_sinkhorn(B, N, d_demand, iters, smooth, scale_bits, d_scaled, d_fixed, d_stretch, d_row_err,
+                               d_status, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_sinkhorn_durations(int B, int k_stride, const int32_t* d_coef, const int32_t* d_count,
+                                const double* d_stretch, int scale_bits, int32_t* d_dur, void* stream) {
+  if (B < 0 || k_stride < 1 || scale_bits < 1 || scale_bits > 24) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_coef || !d_count || !d_stretch || !d_dur) return MOESCHED_EINVAL;
+  if (!aligned4(d_coef) || !aligned4(d_count) || !aligned4(d_dur) || !aligned8(d_stretch)) return MOESCHED_EINVAL;
+  cudaError_t e = run_sinkhorn_durations(B, k_stride, d_coef, d_count, d_stretch, scale_bits, d_dur,
+                                         static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
 int moesched_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* moesched_strerror(int code) {

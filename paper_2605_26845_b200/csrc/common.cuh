@@ -786,6 +786,12 @@ bool model_in_range(const moesched_model_t& m);
 cudaError_t run_ideal_a2a(int B, int N, const int32_t* demand, const moesched_model_t& model, long long* comm_ns,
                           long long* makespan_ns, int32_t* status, cudaStream_t stream);
 
+cudaError_t run_sinkhorn(int B, int N, const int32_t* demand, int iters, double smooth, int scale_bits,
+                         double* scaled, int32_t* fixed, double* stretch, double* row_err, int32_t* status,
+                         cudaStream_t stream);
+cudaError_t run_sinkhorn_durations(int B, int k_stride, const int32_t* coef, const int32_t* count,
+                                   const double* stretch, int scale_bits, int32_t* dur, cudaStream_t stream);
+
 // Launch helper shared by the three kernels.
 template <typename Kernel, typename... Args>
 cudaError_t launch_warp_kernel(Kernel kern, const Geometry& ge, int B, cudaStream_t stream, Args... args) {
