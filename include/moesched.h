@@ -246,10 +246,10 @@ int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_mod
  * its coefficients into token counts with moesched_sinkhorn_durations, and score the result
  * against the ORIGINAL demand with moesched_schedule_eval.
  *
- * The paper fixes no constants; the steps are: X = D + smooth; one sweep divides every row of X
- * by its sum and then every column by its sum; `iters` sweeps. IEEE double arithmetic, row sums
- * accumulated left to right and column sums top to bottom, one rounding per operation -- the
- * result is therefore reproducible bit for bit.
+ * The paper fixes no constants; the steps are: X = D + smooth; one sweep multiplies every row of
+ * X by the reciprocal of its sum and then every column by the reciprocal of its sum; `iters`
+ * sweeps. IEEE double arithmetic, row sums accumulated left to right and column sums top to
+ * bottom, one rounding per operation -- the result is therefore reproducible bit for bit.
  *   d_scaled[b]  = X after the last sweep (column sums 1 up to rounding)
  *   d_row_err[b] = max_i |sum_j scaled[b][i][j] - 1|, the distance from double stochasticity
  *   d_fixed[b]   = floor(scaled * 2^scale_bits + 0.5), the integer matrix for the exact

@@ -595,9 +595,10 @@ int oracle_ideal_a2a(int B, int N, const int32_t* demand, const int64_t* model, 
 // Sinkhorn-Knopp scaling [Sec. 3.1: the preprocessing the paper names for making a demand matrix
 // doubly stochastic before the Birkhoff-von Neumann decomposition]. The paper gives no constants,
 // so the steps are spelled out here: X = D + smooth (smooth > 0 gives every pair a little mass, so
-// that zero rows and columns can be scaled at all); one sweep divides every row by its sum, then
-// every column by its sum; `iters` sweeps. All arithmetic is IEEE double, sums run left to right
-// (rows) and top to bottom (columns), one rounding per operation.
+// that zero rows and columns can be scaled at all); one sweep multiplies every row by the
+// reciprocal of its sum, then every column by the reciprocal of its sum (the usual statement of
+// the iteration: u = 1 / (X v), v = 1 / (X^T u)); `iters` sweeps. All arithmetic is IEEE double,
+// sums run left to right (rows) and top to bottom (columns), one rounding per operation.
 //   scaled   = the matrix after the last sweep (column sums 1 up to rounding, row sums 1 + row_err);
 //   fixed    = round-half-up(scaled * 2^scale_bits): the integer matrix handed to the exact
 //              Birkhoff decomposition (its padding absorbs the rounding residue);
@@ -628,13 +629,15 @@ int oracle_sinkhorn_scale(int B, int N, const int32_t* demand, int iters, double
         double r = 0.0;
         for (int j = 0; j < N; ++j) r = r + S[i * N + j];
         if (!(r > 0.0)) bad = true;
-        for (int j = 0; j < N; ++j) S[i * N + j] = S[i * N + j] / r;
+        const double u = 1.0 / r;
+        for (int j = 0; j < N; ++j) S[i * N + j] = S[i * N + j] * u;
       }
       for (int j = 0; j < N; ++j) {
         double c = 0.0;
         for (int i = 0; i < N; ++i) c = c + S[i * N + j];
         if (!(c > 0.0)) bad = true;
-        for (int i = 0; i < N; ++i) S[i * N + j] = S[i * N + j] / c;
+        const double v = 1.0 / c;
+        for (int i = 0; i < N; ++i) S[i * N + j] = S[i * N + j] * v;
       }
     }
     if (bad) {

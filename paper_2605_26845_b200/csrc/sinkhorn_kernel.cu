@@ -1,16 +1,19 @@
 // Sinkhorn-Knopp scaling (the preprocessing paper Sec. 3.1 names for the Birkhoff-von Neumann
 // decomposition), one warp per demand matrix, IEEE double throughout.
 //
-// X = D + smooth; one sweep divides every row by its sum, then every column by its sum. The
-// sums are defined left to right (rows) and top to bottom (columns) with one rounding per
-// operation, so that the result does not depend on how the work is spread over lanes:
+// X = D + smooth; one sweep multiplies every row by the reciprocal of its sum, then every column
+// by the reciprocal of its sum. The sums are defined left to right (rows) and top to bottom
+// (columns) with one rounding per operation, so that the result does not depend on how the work
+// is spread over lanes:
 //   * a column sum is accumulated by the lane that owns the column (column c: lane c % 32) while
 //     the warp walks the rows from the top -- coalesced loads, sequential order;
 //   * a row sum is accumulated by the lane that owns the row of the current block of 32 rows: the
 //     warp loads 32 x 32 tiles with coalesced row loads into shared memory (row stride 33, no
 //     bank conflicts) and every lane then adds its row's 32 entries in order.
-// The matrix lives in the caller's `scaled` buffer (global memory, L2-resident while a matrix is
-// worked on); the pending division of one pass is applied while the next pass reads the matrix,
+// Up to N = 64 the matrix stays in shared memory for the whole call (32 KB of doubles per warp) and
+// global memory sees the demand once on the way in and the results once on the way out; above
+// that it lives in the caller's `scaled` buffer (global memory, L2-resident while a matrix is
+// worked on). The pending column scaling of one pass is applied while the next pass reads the matrix,
 // so that a sweep costs two reads and two writes of the matrix. Every arithmetic step uses the
 // round-to-nearest intrinsics, which also keeps the compiler from fusing multiplies and adds.
 #include "common.cuh"
@@ -22,10 +25,10 @@ namespace {
 constexpr int SK_TILE = 32 * 33;          // doubles of the tile
 constexpr int SK_WARP = SK_TILE + 256;    // plus one row sum per row
 
-// Applies the pending column division (divide entry (r, c) by col_div of its column) if HAVE_DIV,
-// writes the divided entries back, and leaves in rsum[r] (shared memory) the sum of row r, left to right.
-template <int CPL, bool HAVE_DIV>
-__device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double* tile, const double (&col_div)[CPL],
+// Applies the pending column scaling (entry (r, c) times col_mul of its column) if HAVE_MUL, writes
+// the scaled entries back, and leaves in rsum[r] (shared memory) the sum of row r, left to right.
+template <int CPL, bool HAVE_MUL>
+__device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double* tile, const double (&col_mul)[CPL],
                                               double* rsum) {
   for (int rb = 0; rb * 32 < N; ++rb) {
     double acc = 0.0;
@@ -38,8 +41,8 @@ __device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double
           double v = 0.0;
           if (r < N && c < N) {
             v = S[(size_t)r * N + c];
-            if (HAVE_DIV) {
-              v = __ddiv_rn(v, col_div[cb]);
+            if (HAVE_MUL) {
+              v = __dmul_rn(v, col_mul[cb]);
               S[(size_t)r * N + c] = v;
             }
           }
@@ -58,7 +61,7 @@ __device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double
 
 }  // namespace
 
-template <int CPL>
+template <int CPL, bool RESIDENT>
 __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32_t* __restrict__ demand, int iters,
                                                        double smooth, double scale, double* __restrict__ scaled,
                                                        int32_t* __restrict__ fixed, double* __restrict__ stretch,
@@ -70,7 +73,9 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
   double* tile = reinterpret_cast<double*>(smem_raw) + (size_t)warp * SK_WARP;
   double* rsum = tile + SK_TILE;
   const int32_t* D = demand + (size_t)b * N * N;
-  double* S = scaled + (size_t)b * N * N;
+  double* Sout = scaled + (size_t)b * N * N;
+  double* S = RESIDENT ? reinterpret_cast<double*>(smem_raw) + (size_t)(blockDim.x >> 5) * SK_WARP + (size_t)warp * N * N
+                       : Sout;
   int32_t* Q = fixed + (size_t)b * N * N;
 
   int bad = 0;
@@ -82,17 +87,21 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
   bad = __any_sync(FULL, bad);
   __syncwarp();
 
-  double col_div[CPL];
+  double col_mul[CPL];
 #pragma unroll
-  for (int s = 0; s < CPL; ++s) col_div[s] = 1.0;
+  for (int s = 0; s < CPL; ++s) col_mul[s] = 1.0;
   for (int it = 0; it < iters && !bad; ++it) {
-    if (it == 0) row_sums_pass<CPL, false>(N, lane, S, tile, col_div, rsum);
-    else row_sums_pass<CPL, true>(N, lane, S, tile, col_div, rsum);
+    if (it == 0) row_sums_pass<CPL, false>(N, lane, S, tile, col_mul, rsum);
+    else row_sums_pass<CPL, true>(N, lane, S, tile, col_mul, rsum);
     // a row without mass cannot be scaled
     int zero = 0;
     for (int r = lane; r < N; r += 32) zero |= !(rsum[r] > 0.0);
     if (__any_sync(FULL, zero)) { bad = 1; break; }
-    // divide the rows and accumulate the column sums from the top
+    // each lane turns the sums of its rows into reciprocals
+    __syncwarp();
+    for (int r = lane; r < N; r += 32) rsum[r] = __ddiv_rn(1.0, rsum[r]);
+    __syncwarp();
+    // scale the rows and accumulate the column sums from the top
     double csum[CPL];
 #pragma unroll
     for (int s = 0; s < CPL; ++s) csum[s] = 0.0;
@@ -102,7 +111,7 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
       for (int s = 0; s < CPL; ++s) {
         const int c = s * 32 + lane;
         if (c < N) {
-          const double v = __ddiv_rn(S[(size_t)r * N + c], rv);
+          const double v = __dmul_rn(S[(size_t)r * N + c], rv);
           S[(size_t)r * N + c] = v;
           csum[s] = __dadd_rn(csum[s], v);
         }
@@ -112,7 +121,7 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
 #pragma unroll
     for (int s = 0; s < CPL; ++s) {
       if (s * 32 + lane < N) zero |= !(csum[s] > 0.0);
-      col_div[s] = csum[s];
+      col_mul[s] = __ddiv_rn(1.0, csum[s]);
     }
     if (__any_sync(FULL, zero)) { bad = 1; break; }
     __syncwarp();
@@ -120,20 +129,22 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
 
   if (bad) {
     __syncwarp();
-    for (int e = lane; e < N * N; e += 32) { S[e] = 0.0; Q[e] = 0; }
+    for (int e = lane; e < N * N; e += 32) { Sout[e] = 0.0; Q[e] = 0; }
     if (lane == 0) { stretch[b] = 0.0; row_err[b] = 0.0; status[b] = MOESCHED_ST_BAD_INPUT; }
     return;
   }
 
-  // the last column division, the row sums of the result, the fixed-point matrix and the stretch
-  row_sums_pass<CPL, true>(N, lane, S, tile, col_div, rsum);
+  // the last column scaling, the row sums of the result, the fixed-point matrix and the stretch
+  row_sums_pass<CPL, true>(N, lane, S, tile, col_mul, rsum);
   double err = 0.0;
   for (int r = lane; r < N; r += 32) err = fmax(err, fabs(__dadd_rn(rsum[r], -1.0)));
   __syncwarp();
   double st = 0.0;
   int dropped = 0;
   for (int e = lane; e < N * N; e += 32) {
-    const double q = floor(__dadd_rn(__dmul_rn(S[e], scale), 0.5));
+    const double v = S[e];
+    if (RESIDENT) Sout[e] = v;
+    const double q = floor(__dadd_rn(__dmul_rn(v, scale), 0.5));
     const int qi = (int)q;
     Q[e] = qi;
     const int d = D[e];
@@ -175,22 +186,24 @@ __global__ void __launch_bounds__(256) sinkhorn_durations_kernel(int B, int k_st
 cudaError_t run_sinkhorn(int B, int N, const int32_t* demand, int iters, double smooth, int scale_bits,
                          double* scaled, int32_t* fixed, double* stretch, double* row_err, int32_t* status,
                          cudaStream_t stream) {
-  const int wpb = 4;
-  const size_t smem = (size_t)wpb * SK_WARP * sizeof(double);
+  const bool resident = N <= 64;
+  const int wpb = resident ? 1 : 4;
+  const size_t smem = (size_t)wpb * (SK_WARP + (resident ? N * N : 0)) * sizeof(double);
   const double scale = (double)(1 << scale_bits);
   const int grid = (B + wpb - 1) / wpb;
-#define MOESCHED_GO(C)                                                                                            \
-  do {                                                                                                            \
-    cudaError_t e = cudaFuncSetAttribute(sinkhorn_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-    if (e != cudaSuccess) return e;                                                                               \
-    sinkhorn_kernel<C><<<grid, 32 * wpb, smem, stream>>>(B, N, demand, iters, smooth, scale, scaled, fixed, stretch, \
-                                                         row_err, status);                                        \
-    return cudaGetLastError();                                                                                    \
+#define MOESCHED_GO(C, R)                                                                                           \
+  do {                                                                                                              \
+    cudaError_t e = cudaFuncSetAttribute(sinkhorn_kernel<C, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                         (int)smem);                                                                \
+    if (e != cudaSuccess) return e;                                                                                 \
+    sinkhorn_kernel<C, R><<<grid, 32 * wpb, smem, stream>>>(B, N, demand, iters, smooth, scale, scaled, fixed,      \
+                                                            stretch, row_err, status);                              \
+    return cudaGetLastError();                                                                                      \
   } while (0)
-  if (N <= 32) MOESCHED_GO(1);
-  if (N <= 64) MOESCHED_GO(2);
-  if (N <= 128) MOESCHED_GO(4);
-  MOESCHED_GO(8);
+  if (N <= 32) MOESCHED_GO(1, true);
+  if (N <= 64) MOESCHED_GO(2, true);
+  if (N <= 128) MOESCHED_GO(4, false);
+  MOESCHED_GO(8, false);
 #undef MOESCHED_GO
 }
 

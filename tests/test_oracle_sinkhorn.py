@@ -64,14 +64,14 @@ def test_against_a_vectorised_statement_and_sweep_by_sweep_error():
 
 def test_balanced_inputs_and_power_of_two_invariance():
     N = 8                                                # 1/8 is exact in binary floating point
-    J = np.full((1, N, N), 7, np.int32)
+    J = np.full((1, N, N), 8, np.int32)
     r = oracle.sinkhorn_scale(J, 1, 0.0, 20)
     assert (r["scaled"] == 1.0 / N).all() and r["row_err"][0] < 1e-15
     P = np.zeros((1, N, N), np.int32)
-    P[0, np.arange(N), np.roll(np.arange(N), 2)] = 12
+    P[0, np.arange(N), np.roll(np.arange(N), 2)] = 16
     r = oracle.sinkhorn_scale(P, 3, 0.0, 20)
     assert (r["scaled"][0] == (P[0] > 0)).all()
-    assert (r["fixed"][0] == (P[0] > 0) * 2**20).all() and r["stretch"][0] == 12.0
+    assert (r["fixed"][0] == (P[0] > 0) * 2**20).all() and r["stretch"][0] == 16.0
     D = random_matrices(2, 9, seed=3, kind="uniform", high=100)
     a = oracle.sinkhorn_scale(D, 7, 0.5, 16)
     b = oracle.sinkhorn_scale(D * 4, 7, 2.0, 16)        # scaling by a power of two is exact in binary floating point
