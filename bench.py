@@ -334,11 +334,12 @@ def main():
 
     # ---- Sinkhorn-Knopp scaling (the paper's preprocessing for BvN; not part of the step either) ----
     sk_ms = []
+    sk = ms.sinkhorn_scale(d, SINKHORN_ITERS, 0.5, 20)          # allocates the outputs once, untimed
     for _ in range(3):
         flush.fill_(1)
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record(stream)
-        sk = ms.sinkhorn_scale(d, SINKHORN_ITERS, 0.5, 20)
+        ms.sinkhorn_scale(d, SINKHORN_ITERS, 0.5, 20, out=sk)
         a1.record(stream)
         a1.synchronize()
         sk_ms.append(a0.elapsed_time(a1))

@@ -199,18 +199,24 @@ def probe_int_rate(device=None, blocks=148 * 8, iters=20000, reps=3) -> float:
     return best
 
 
-def sinkhorn_scale(demand, iters=20, smooth=0.5, scale_bits=20) -> dict:
+def sinkhorn_scale(demand, iters=20, smooth=0.5, scale_bits=20, out=None) -> dict:
     """Sinkhorn-Knopp scaling of a batch (paper Sec. 3.1). Returns scaled [B, N, N] float64, fixed
     [B, N, N] int32 (= round(scaled * 2^scale_bits), the input of bvn_decompose), stretch [B], row_err [B]
-    float64 and status [B]."""
+    float64 and status [B]; `out` may hand back the dict of an earlier call of the same shape for reuse."""
     demand = _check_demand(demand)
     B, N, _ = demand.shape
     dev = demand.device
-    out = dict(scaled=torch.empty((B, N, N), dtype=torch.float64, device=dev),
-               fixed=torch.empty((B, N, N), dtype=torch.int32, device=dev),
-               stretch=torch.empty(B, dtype=torch.float64, device=dev),
-               row_err=torch.empty(B, dtype=torch.float64, device=dev),
-               status=torch.empty(B, dtype=torch.int32, device=dev))
+    if out is None:
+        out = dict(scaled=torch.empty((B, N, N), dtype=torch.float64, device=dev),
+                   fixed=torch.empty((B, N, N), dtype=torch.int32, device=dev),
+                   stretch=torch.empty(B, dtype=torch.float64, device=dev),
+                   row_err=torch.empty(B, dtype=torch.float64, device=dev),
+                   status=torch.empty(B, dtype=torch.int32, device=dev))
+    else:
+        _dev(out["scaled"], torch.float64, "out['scaled']")
+        _dev(out["fixed"], torch.int32, "out['fixed']")
+        if out["scaled"].shape != demand.shape or out["fixed"].shape != demand.shape:
+            raise MoeschedError("out has the wrong shape")
     rc = load_library().moesched_sinkhorn_scale(B, N, _ptr(demand), int(iters), ctypes.c_double(float(smooth)),
                                                 int(scale_bits), _ptr(out["scaled"]), _ptr(out["fixed"]),
                                                 _ptr(out["stretch"]), _ptr(out["row_err"]), _ptr(out["status"]),
