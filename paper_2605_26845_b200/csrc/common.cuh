@@ -770,6 +770,10 @@ cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm
                    int32_t* residual, int32_t* status, long long* work, cudaStream_t stream);
 cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
                     int32_t* aug, int32_t* scratch, int32_t* status, long long* work, cudaStream_t stream);
+// the same decomposition with one CTA of several warps per matrix (scratch required, 64 < N <= 256)
+cudaError_t run_bvn_team(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef,
+                         int32_t* count, int32_t* aug, int32_t* scratch, int32_t* status, long long* work,
+                         cudaStream_t stream);
 // row stride (ints) of the global working copy used by the Birkhoff kernel
 inline int bvn_scratch_stride(int N) { return (N + 7) / 8 * 8; }
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,

@@ -1,0 +1,312 @@
+// Building blocks for the kernels in which a TEAM of NW warps (one CTA) owns one demand matrix.
+// They serve batches with too few matrices to fill the SMs with one warp per matrix (N > 128 in
+// the benchmarked configurations). Thread t of the CTA owns row t and column t of the matrix: its
+// adjacency to the columns (Rr) and to the rows (Cc) as bit masks of W = NW words in registers, its
+// matched column and row as scalars. Sets of rows or columns that all threads need are built in
+// shared memory with one atomic per member and read back after a CTA barrier; membership that
+// only the owner needs stays a flag in the owner's registers. Every value a branch depends on is
+// read from shared memory after a barrier, so control flow is uniform across the CTA and every
+// barrier is reached by all of its threads.
+#pragma once
+
+#include "common.cuh"
+
+namespace moesched {
+
+// Reduction slots in shared memory, three deep so that one barrier per phase is enough: in phase p
+// the threads clear the slot of phase p+1 (last read before the barrier of phase p-1), add to the
+// slot of phase p, meet at the barrier and read the slot of phase p.
+struct TeamRed {
+  static constexpr int SET = 0;    // words 0..7: a set of rows or columns (bitwise OR)
+  static constexpr int MIN = 8;    // unsigned minimum (starts at 0xffffffff)
+  static constexpr int ADD = 9;    // sum
+  static constexpr int MAX = 10;   // unsigned maximum
+  static constexpr int SLOT = 12;
+  unsigned* buf;   // 3 * SLOT words
+  int which;       // slot of the current phase: 0, 1, 2 (uniform)
+
+  __device__ __forceinline__ void init(unsigned* shared_words) {
+    buf = shared_words;
+    which = 0;
+    if (threadIdx.x < 3 * SLOT) buf[threadIdx.x] = (threadIdx.x % SLOT) == MIN ? 0xffffffffu : 0u;
+    __syncthreads();
+  }
+  __device__ __forceinline__ unsigned* cur() const { return buf + which * SLOT; }
+  // start of a phase: clear the slot the next phase will use
+  __device__ __forceinline__ void open() const {
+    const int nx = which == 2 ? 0 : which + 1;
+    if (threadIdx.x < SLOT) buf[nx * SLOT + threadIdx.x] = threadIdx.x == MIN ? 0xffffffffu : 0u;
+  }
+  // all contributions made: after this the slot may be read
+  __device__ __forceinline__ void close() const { __syncthreads(); }
+  // the slot has been read
+  __device__ __forceinline__ void next() { which = which == 2 ? 0 : which + 1; }
+
+  // member `index` joins the set if flag; a warp with many joiners combines them first
+  template <int W>
+  __device__ __forceinline__ void add_member(bool flag, int index, int lane) const {
+    const unsigned ball = __ballot_sync(FULL, flag);
+    if (ball == 0u) return;
+    unsigned* s = cur() + SET;
+    if (__popc(ball) <= 4) {
+      if (flag) atomicOr(&s[index >> 5], 1u << (index & 31));
+    } else {
+      unsigned mine = 0u;
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        const unsigned r = __reduce_or_sync(FULL, flag ? onehot_word(index, w) : 0u);
+        if (lane == w) mine = r;
+      }
+      if (lane < W && mine != 0u) atomicOr(&s[lane], mine);
+    }
+  }
+  template <int W>
+  __device__ __forceinline__ void read_set(unsigned (&out)[W]) const {
+#pragma unroll
+    for (int w = 0; w < W; ++w) out[w] = cur()[SET + w];
+  }
+  // lowest index among the flagged threads, packed with a 16-bit payload: index << 16 | payload
+  __device__ __forceinline__ void min_key(bool flag, int index, int payload, int lane) const {
+    const unsigned ball = __ballot_sync(FULL, flag);
+    if (ball == 0u) return;
+    if (lane == __ffs(ball) - 1) atomicMin(&cur()[MIN], ((unsigned)index << 16) | ((unsigned)payload & 0xffffu));
+  }
+  __device__ __forceinline__ void max_val(bool flag, unsigned v, int lane) const {
+    const unsigned m = __reduce_max_sync(FULL, flag ? v : 0u);
+    if (lane == 0 && m != 0u) atomicMax(&cur()[MAX], m);
+  }
+  __device__ __forceinline__ void add_val(unsigned v, int lane) const {
+    const unsigned m = __reduce_add_sync(FULL, v);
+    if (lane == 0 && m != 0u) atomicAdd(&cur()[ADD], m);
+  }
+};
+
+template <int NW>
+struct TeamShared {
+  static constexpr int NT = 32 * NW;
+  short x[NT];            // row -> column (-1: none)
+  short mr[NT];           // column -> row (-1: none)
+  short par[NT];          // augmenting search: row from which a column was reached
+  int lvl[NT];            // stamp of the backward-search level at which a row was reached
+  unsigned red[3 * TeamRed::SLOT];
+  unsigned tot[NW * NW];  // per-warp column sets of the candidate test
+  unsigned ri[NW];        // columns adjacent to the row being searched
+  int misc[8];
+};
+
+template <int W>
+__device__ __forceinline__ bool meets(const unsigned (&a)[W], const unsigned (&b)[W]) {
+  unsigned o = 0u;
+#pragma unroll
+  for (int w = 0; w < W; ++w) o |= a[w] & b[w];
+  return o != 0u;
+}
+
+// The matching of one team: who is matched to whom, as the owner thread sees it.
+template <int NW>
+struct TeamMatch {
+  static constexpr int W = NW;
+  unsigned Rr[W];   // columns adjacent to row t
+  unsigned Cc[W];   // rows adjacent to column t
+  int my_x;         // column of row t (-1: free)
+  int my_mr;        // row of column t (-1: free)
+};
+
+// Rows that could move to a lower column: row r qualifies iff it is adjacent to a column below its
+// own whose row lies above r. The columns matched to rows above r are an exclusive suffix OR over
+// the threads: inside the warp by shuffles, across warps through shared memory. One barrier.
+template <int NW>
+__device__ __forceinline__ bool team_is_candidate(TeamShared<NW>& sh, int t, int lane, int warp, bool in,
+                                                  const TeamMatch<NW>& m) {
+  constexpr int W = NW;
+  unsigned v[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) v[w] = in ? onehot_word(m.my_x, w) : 0u;
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned u = __shfl_down_sync(FULL, v[w], o);
+      if (lane + o < 32) v[w] |= u;
+    }
+  }
+  unsigned above[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    const unsigned u = __shfl_down_sync(FULL, v[w], 1);
+    above[w] = lane < 31 ? u : 0u;
+    const unsigned total = __shfl_sync(FULL, v[w], 0);
+    if (lane == w) sh.tot[warp * W + w] = total;
+  }
+  __syncthreads();
+  for (int g = warp + 1; g < NW; ++g) {
+#pragma unroll
+    for (int w = 0; w < W; ++w) above[w] |= sh.tot[g * W + w];
+  }
+  if (!in || m.my_x < 0) return false;
+  unsigned o = 0u;
+#pragma unroll
+  for (int w = 0; w < W; ++w) o |= m.Rr[w] & above[w] & ~ge_word(m.my_x, w);
+  return o != 0u;
+}
+
+// Memo carried from one call of team_canonicalise to the next when the graph only loses edges
+// between calls (Birkhoff), the counterpart of CanonMemo in common.cuh spread over the row owners:
+// known = row t's last search found no lower column and none of the rows that could reach it has
+// changed column since; dep = the searched rows whose recorded set contains row t; changed = row
+// t's column changed since the last call.
+template <int NW>
+struct TeamMemo {
+  bool known, changed;
+  unsigned dep[NW];
+  __device__ __forceinline__ void reset() {
+    known = changed = false;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) dep[w] = 0u;
+  }
+};
+
+// One phase: the rows flagged `moved` void every record that contains them (and their own).
+template <int NW>
+__device__ __forceinline__ void team_void_records(TeamRed& red, int t, bool moved, TeamMemo<NW>& memo) {
+  constexpr int W = NW;
+  red.open();
+  if (moved) {
+    unsigned* s = red.cur() + TeamRed::SET;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const unsigned v = memo.dep[w] | onehot_word(t, w);
+      if (v != 0u) atomicOr(&s[w], v);
+      memo.dep[w] = 0u;
+    }
+  }
+  red.close();
+  if ((red.cur()[TeamRed::SET + (t >> 5)] >> (t & 31)) & 1u) memo.known = false;
+  red.next();
+}
+
+// Lexicographically smallest perfect matching of the graph (Rr / Cc) over the window of rows
+// [start, last], given a perfect matching that already equals the answer below `start` (see
+// canonicalise() in common.cuh for the argument; this is the same procedure with the sets spread
+// over the CTA). For each row i that could move: the rows >= i that reach i by alternating steps
+// are found level by level -- a row joins when it is adjacent to the column of a row of the
+// previous level -- then row i takes the lowest adjacent column whose row was reached and the
+// matching is rotated along the cycle. Returns false if an iteration limit was hit. Uniform.
+template <int NW, bool MEMO>
+__device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& red, int N, int t, int lane, int warp,
+                                                  bool in, TeamMatch<NW>& m, TeamMemo<NW>& memo, int& stamp,
+                                                  int start, int last, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = NW;
+  bool ok_all = true;
+  if constexpr (MEMO) {
+    team_void_records<NW>(red, t, memo.changed, memo);
+    memo.changed = false;
+  }
+  bool cand = team_is_candidate<NW>(sh, t, lane, warp, in, m);
+  int from = start;
+  for (int guard = 0; guard < N; ++guard) {
+    // next row that could move
+    red.open();
+    red.min_key(cand && t >= from && t <= last && !(MEMO && memo.known), t, 0, lane);
+    red.close();
+    const unsigned ikey = red.cur()[TeamRed::MIN];
+    red.next();
+    if (ikey == 0xffffffffu) break;
+    const int i = (int)(ikey >> 16);
+    from = i + 1;
+    if (t == 0) work[WK_SWEEP]++;
+    stamp += N + 2;
+    // level 0: row i itself. Its adjacency is published for the column choice (read several
+    // barriers later; the previous search's readers are past the barrier above).
+    bool in_anc = t == i;
+    if (t == i) {
+      sh.lvl[i] = stamp;
+#pragma unroll
+      for (int w = 0; w < W; ++w) sh.ri[w] = m.Rr[w];
+    }
+    const int xi = sh.x[i];
+    unsigned xf[W];   // columns of the rows of the current level
+#pragma unroll
+    for (int w = 0; w < W; ++w) xf[w] = onehot_word(xi, w);
+    int level = 0;
+    for (int it = 0; it < N; ++it) {
+      red.open();
+      const bool isnew = in && t > i && !in_anc && meets<W>(m.Rr, xf);
+      if (isnew) {
+        in_anc = true;
+        sh.lvl[t] = stamp + level + 1;
+      }
+      red.add_member<W>(isnew, m.my_x, lane);
+      red.close();
+      red.read_set<W>(xf);
+      red.next();
+      if (t == 0) work[WK_LEVEL]++;
+      if (!any_bit<W>(xf)) break;
+      ++level;
+    }
+    // lowest column row i may take: adjacent to i, its row reached (its own column always qualifies)
+    red.open();
+    {
+      const bool adj = in && ((sh.ri[t >> 5] >> (t & 31)) & 1u);
+      const bool reached = adj && m.my_mr >= 0 && sh.lvl[m.my_mr] >= stamp;
+      red.min_key(reached, t, m.my_mr, lane);
+    }
+    red.close();
+    const unsigned key = red.cur()[TeamRed::MIN];
+    red.next();
+    if (key == 0xffffffffu) { ok_all = false; continue; }
+    const int jstar = (int)(key >> 16);
+    if (jstar == xi) {
+      // record: row i stays put until one of the rows that can reach it changes column
+      if constexpr (MEMO) {
+        if (in_anc) {
+#pragma unroll
+          for (int w = 0; w < W; ++w) memo.dep[w] |= onehot_word(i, w);
+        }
+        if (t == i) memo.known = true;
+      }
+      continue;
+    }
+    // rotate along the alternating cycle: the row that gives up column jstar takes the column of
+    // its successor towards row i, and so on down the levels
+    int cur = (int)(key & 0xffffu);
+    int lvl = sh.lvl[cur] - stamp;
+    if (lvl <= 0 || lvl > level) { ok_all = false; continue; }
+    for (int it = 0; it < N && lvl > 0; ++it) {
+      red.open();
+      const bool q = in && m.my_mr >= 0 && sh.lvl[m.my_mr] == stamp + lvl - 1 && test_bit<W>(m.Cc, cur);
+      red.min_key(q, t, m.my_mr, lane);
+      red.close();
+      const unsigned k2 = red.cur()[TeamRed::MIN];
+      red.next();
+      if (k2 == 0xffffffffu) { ok_all = false; break; }
+      const int c2 = (int)(k2 >> 16), nxt = (int)(k2 & 0xffffu);
+      if (t == c2) {
+        m.my_mr = cur;
+        sh.mr[c2] = (short)cur;
+        sh.x[cur] = (short)c2;
+      }
+      last = max(last, cur);
+      cur = nxt;
+      --lvl;
+      if (t == 0) work[WK_ROT]++;
+    }
+    if (t == jstar) {
+      m.my_mr = i;
+      sh.mr[jstar] = (short)i;
+      sh.x[i] = (short)jstar;
+    }
+    __syncthreads();
+    {
+      const int nx = sh.x[t];
+      const bool moved = nx != m.my_x;
+      m.my_x = nx;
+      // the moved rows changed column: every record that contains one of them is void
+      if constexpr (MEMO) team_void_records<NW>(red, t, moved, memo);
+    }
+    cand = team_is_candidate<NW>(sh, t, lane, warp, in, m);
+  }
+  return ok_all;
+}
+
+}  // namespace moesched

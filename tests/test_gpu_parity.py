@@ -70,6 +70,22 @@ def test_large_matrices_prefix(N, kw):
     check_all(D, 6, 10)
 
 
+@pytest.mark.parametrize("N,kw", [(129, KINDS[0]), (200, KINDS[2]), (256, KINDS[0]), (256, KINDS[1])])
+def test_team_kernel_deep_prefix(N, kw):
+    """Above 128 ranks a small batch runs the Birkhoff kernel that puts a CTA of eight warps on each
+    matrix: several hundred matchings deep against the oracle, and against the one-warp kernel
+    (shared-memory placement) on the same inputs."""
+    D = random_matrices(2, N, seed=7000 + N, **kw)
+    d = dev(D)
+    K = 400
+    rv = oracle.bvn_decompose(D, K, threads=8)
+    team = ms.bvn_decompose(d, K, want_aug=True, scratch=True)
+    warp = ms.bvn_decompose(d, K, want_aug=True, scratch=False)
+    for v in (team, warp):
+        assert_schedule_equal(v, rv, "coef")
+        assert (v.extra.cpu().numpy() == rv["aug"]).all()
+
+
 @pytest.mark.parametrize("N", [1, 2, 5, 8, 17, 64, 100])
 def test_closed_form_cases(N):
     cases = structured_cases(N, m=7)
