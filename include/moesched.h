@@ -112,7 +112,8 @@ typedef struct moesched_model {
  *                   0 shortest-path column scans, 1 augmentations, 2 rows
  *                   tried against their best column, 3 canonicalisation
  *                   sweeps that searched, 4 search levels, 5 rotation steps,
- *                   6 matchings, 7 unused
+ *                   6 matchings, 7 rows matched along tight edges before the
+ *                   shortest-path phase
  */
 int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                           int32_t* d_dur, int32_t* d_count, int32_t* d_residual,

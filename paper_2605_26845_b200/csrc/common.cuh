@@ -748,6 +748,94 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
   return ok_all;
 }
 
+// ---- augmenting search on a 0/1 graph --------------------------------------------------------
+// Augmenting search from free row f over alternating paths of the graph C (the support graph of
+// the Birkhoff step, the tight edges of a greedy step).
+// Among all augmenting paths it takes one whose lowest row is as high as possible: the
+// search first uses only rows >= t = f and lowers t to the highest waiting row only when
+// it is stuck, so the rows below the returned path keep their columns. [lo, hi] is widened
+// to cover every row whose column changed. Returns false when no augmenting path exists
+// (cannot happen for a balanced matrix).
+template <int CPL>
+__device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsigned (&C)[CPL][CPL], Match<CPL>& M,
+                                             short* x, int& lo, int& hi, unsigned (&changed)[CPL],
+                                             unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = CPL;
+  unsigned F[W], P[W];   // frontier rows; rows met but still below the threshold
+#pragma unroll
+  for (int w = 0; w < W; ++w) F[w] = P[w] = 0u;
+  set_bit<W>(F, f);
+  int t = f;
+  unsigned visited = 0u;
+  int par[CPL];
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) par[s] = -1;
+  int jf = -1;
+  for (int it = 0; it < 2 * N + 2; ++it) {
+    unsigned met[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) met[w] = 0u;
+    int freeslot = -1;
+#pragma unroll
+    for (int ss = 0; ss < CPL; ++ss) {
+      const int s = CPL - 1 - ss;
+      if (!((visited >> s) & 1u)) {
+        unsigned hit[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) hit[w] = C[s][w] & F[w];
+        if (any_bit<W>(hit)) {
+          visited |= 1u << s;
+          par[s] = lowest_bit<W>(hit);
+          if (M.mr[s] < 0) freeslot = s;
+          else M.add_to(met, s);
+        }
+      }
+    }
+    work[WK_SCAN]++;
+    const unsigned fb = __ballot_sync(FULL, freeslot >= 0);
+    if (fb) {
+      const int L = __ffs(fb) - 1;
+      jf = L * CPL + __shfl_sync(FULL, freeslot, L);
+      break;
+    }
+    bool grew = false;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const unsigned m = __reduce_or_sync(FULL, met[w]);
+      const unsigned ge = ge_word(t, w);
+      F[w] = m & ge;
+      P[w] |= m & ~ge;
+      grew |= F[w] != 0u;
+    }
+    if (!grew) {
+      const int r = highest_bit<W>(P);   // admit the highest waiting row, and only that one
+      if (r < 0) return false;
+      t = r;
+      clear_bit<W>(P, r);
+      set_bit<W>(F, r);
+    }
+  }
+  if (jf < 0) return false;
+  int j = jf;
+  for (int it = 0; it <= N; ++it) {
+    const int L = j / CPL, sl = j % CPL;
+    const int i = __shfl_sync(FULL, pick<CPL>(par, sl), L);
+    const int jprev = x[i];
+    __syncwarp();
+    if (lane == L) M.assign(sl, i);
+    if (lane == 0) x[i] = (short)j;
+    __syncwarp();
+    lo = min(lo, i);
+    hi = max(hi, i);
+    set_bit<W>(changed, i);
+    work[WK_AUG]++;
+    if (i == f) return true;
+    j = jprev;
+    if (j < 0) return false;
+  }
+  return false;
+}
+
 // Time of one expert batch of g tokens (see moesched_model_t).
 __device__ __forceinline__ long long batch_time_ns(const moesched_model_t& m, long long g) {
   if (g <= 0) return 0;
