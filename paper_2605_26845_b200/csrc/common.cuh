@@ -625,29 +625,36 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
     }
   }
   candidate_rows<CPL>(lane, C, M, cand);
-  int from = start;
-  for (int guard = 0; guard < N; ++guard) {
-    // next row that could move and is not covered by a record that still holds:
-    // unrecorded rows up to the last changed row
-    unsigned todo[W];
+  // rows still to be looked at: those that could move, from `start` up to the last changed row,
+  // not covered by a record that still holds. Rebuilt only after a rotation; otherwise the row just
+  // searched is simply struck off.
+  unsigned todo[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) {
-      unsigned need = cand[w] & ge_word(from, w);
-      if constexpr (MEMO) need &= ~memo.known[w] & ~ge_word(last + 1, w);
-      todo[w] = need;
-    }
+  for (int w = 0; w < W; ++w) {
+    unsigned need = cand[w] & ge_word(start, w) & ~ge_word(last + 1, w);
+    if constexpr (MEMO) need &= ~memo.known[w];
+    todo[w] = need;
+  }
+  for (int guard = 0; guard < N; ++guard) {
     const int i = lowest_bit<W>(todo);
-    if (i < 0 || i > last) break;
-    from = i + 1;
+    if (i < 0) break;
     const int xi = x[i];
     work[WK_SWEEP]++;
-    // backward search from row i among the rows >= i
+    // backward search from row i among the rows >= i; the one-hot mask of i and the set {i, i+1, ...}
+    // come from isolating the lowest bit of todo
     unsigned anc[W], F[W], alive[W], imask[W];
+    {
+      bool below = true;   // all lower words of todo are empty
 #pragma unroll
-    for (int w = 0; w < W; ++w) {
-      imask[w] = onehot_word(i, w);
-      anc[w] = F[w] = imask[w];
-      alive[w] = ge_word(i, w);
+      for (int w = 0; w < W; ++w) {
+        const unsigned lowbit = todo[w] & (0u - todo[w]);
+        const bool here = below && todo[w] != 0u;
+        imask[w] = here ? lowbit : 0u;
+        alive[w] = here ? (0u - lowbit) : (below ? 0u : 0xffffffffu);
+        below = below && todo[w] == 0u;
+        todo[w] &= ~imask[w];
+        anc[w] = F[w] = imask[w];
+      }
     }
     int level = 0;
     if (lane < W) hist[lane] = pick<W>(F, lane);
@@ -743,6 +750,12 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         for (int w = 0; w < W; ++w) memo.known[w] &= ~hit[w];
       }
       candidate_rows<CPL>(lane, C, M, cand);
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        unsigned need = cand[w] & ge_word(i + 1, w) & ~ge_word(last + 1, w);
+        if constexpr (MEMO) need &= ~memo.known[w];
+        todo[w] = need;
+      }
     }
   }
   return ok_all;
