@@ -14,7 +14,9 @@ namespace moesched {
 
 // MODE 0: matrix in this CTA's shared memory; 1: split over a 2-CTA cluster; 2: working copy
 // in global memory (scratch), which leaves room for many more warps per SM.
-template <int CPL, int MODE>
+// COUNT: the per-matrix work counters are wanted (they are plain register increments that the
+// compiler drops, registers included, when nothing reads them).
+template <int CPL, int MODE, bool COUNT>
 __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                   uint8_t* __restrict__ perm, int32_t* __restrict__ coef,
                                                   int32_t* __restrict__ count, int32_t* __restrict__ aug,
@@ -198,8 +200,11 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       // unmatch the rows whose entry vanished
       M.release(freerows);
       __syncwarp();
-      for (int r = lane; r < N; r += 32)
-        if (test_bit<W>(freerows, r)) x[r] = -1;
+#pragma unroll
+      for (int q = 0; q < W; ++q) {   // lane l looks after rows l, l + 32, ...
+        const int r = q * 32 + lane;
+        if (r < N && ((freerows[q] >> lane) & 1u)) x[r] = -1;
+      }
       __syncwarp();
     }
     if (st_code == MOESCHED_ST_OK && nnz > 0) st_code = MOESCHED_ST_TRUNCATED;
@@ -210,9 +215,11 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
     count[b] = k;
     status[b] = st_code;
   }
-  if (work_out != nullptr && lane == 0) {
+  if constexpr (COUNT) {
+    if (work_out != nullptr && lane == 0) {
 #pragma unroll
-    for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+      for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+    }
   }
   cluster_epilogue<CLUSTER>();
 }
@@ -222,9 +229,14 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
                     int32_t* aug, int32_t* scratch, int32_t* status, long long* work, cudaStream_t stream) {
   Geometry ge = plan_geometry(N);
-#define MOESCHED_GO(C, M)                                                                                    \
-  return launch_warp_kernel(bvn_kernel<C, M>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, count, \
-                            aug, scratch, status, work)
+#define MOESCHED_GO(C, M)                                                                                     \
+  do {                                                                                                        \
+    if (work != nullptr)                                                                                      \
+      return launch_warp_kernel(bvn_kernel<C, M, true>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, \
+                                count, aug, scratch, status, work);                                           \
+    return launch_warp_kernel(bvn_kernel<C, M, false>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef,  \
+                              count, aug, scratch, status, work);                                             \
+  } while (0)
   // Above 128 ranks a batch that leaves most SMs with a single warp goes to the kernel that puts a
   // CTA of eight warps on each matrix (measured at N = 256, B = 256: 1.0 s against 1.8 s; at N = 128,
   // B = 1024 one warp per matrix is the faster of the two, 0.32 s against 0.46 s).

@@ -779,6 +779,9 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   for (int w = 0; w < W; ++w) F[w] = P[w] = 0u;
   set_bit<W>(F, f);
   int t = f;
+  unsigned at_or_above[W];   // rows >= t
+#pragma unroll
+  for (int w = 0; w < W; ++w) at_or_above[w] = ge_word(t, w);
   unsigned visited = 0u;
   int par[CPL];
 #pragma unroll
@@ -815,7 +818,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
 #pragma unroll
     for (int w = 0; w < W; ++w) {
       const unsigned m = __reduce_or_sync(FULL, met[w]);
-      const unsigned ge = ge_word(t, w);
+      const unsigned ge = at_or_above[w];
       F[w] = m & ge;
       P[w] |= m & ~ge;
       grew |= F[w] != 0u;
@@ -824,6 +827,8 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
       const int r = highest_bit<W>(P);   // admit the highest waiting row, and only that one
       if (r < 0) return false;
       t = r;
+#pragma unroll
+      for (int w = 0; w < W; ++w) at_or_above[w] = ge_word(t, w);
       clear_bit<W>(P, r);
       set_bit<W>(F, r);
     }

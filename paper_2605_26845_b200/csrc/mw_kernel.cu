@@ -212,7 +212,8 @@ __global__ void __launch_bounds__(256) mw_classify_kernel(int B, int N, const in
 
 // MODE 0: matrix in this CTA's shared memory as int32; 1: split over a 2-CTA cluster; 2: 16-bit entries.
 // only_class != 0: handle only the matrices whose status[b] holds that class.
-template <int CPL, int MODE>
+// COUNT: the per-matrix work counters are wanted (register increments the compiler drops otherwise).
+template <int CPL, int MODE, bool COUNT>
 __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                  uint8_t* __restrict__ perm, int32_t* __restrict__ dur,
                                                  int32_t* __restrict__ count, int32_t* __restrict__ residual,
@@ -326,9 +327,11 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
       for (int c = lane; c < N; c += 32) ro[(size_t)r * N + c] = rp[c];
     }
   }
-  if (work_out != nullptr && lane == 0) {
+  if constexpr (COUNT) {
+    if (work_out != nullptr && lane == 0) {
 #pragma unroll
-    for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+      for (int q = 0; q < MOESCHED_WORK_FIELDS; ++q) work_out[(size_t)b * MOESCHED_WORK_FIELDS + q] = work[q];
+    }
   }
   cluster_epilogue<CLUSTER>();
 }
@@ -344,9 +347,14 @@ template <int MODE>
 static cudaError_t launch_mw_mode(Geometry ge, int B, int N, const int32_t* demand, int k_max, uint8_t* perm,
                                   int32_t* dur, int32_t* count, int32_t* residual, int32_t* status, long long* work,
                                   int only_class, cudaStream_t stream) {
-#define MOESCHED_GO(C)                                                                                      \
-  return launch_warp_kernel(mw_kernel<C, MODE>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur, count, \
-                            residual, status, work, only_class)
+#define MOESCHED_GO(C)                                                                                         \
+  do {                                                                                                         \
+    if (work != nullptr)                                                                                       \
+      return launch_warp_kernel(mw_kernel<C, MODE, true>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur, \
+                                count, residual, status, work, only_class);                                    \
+    return launch_warp_kernel(mw_kernel<C, MODE, false>, ge, B, stream, B, N, ge.S, demand, k_max, perm, dur,  \
+                              count, residual, status, work, only_class);                                      \
+  } while (0)
   switch (ge.cpl) {
     case 1: MOESCHED_GO(1);
     case 2: MOESCHED_GO(2);
