@@ -500,20 +500,32 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
     const unsigned t = __shfl_down_sync(FULL, v, 1);
     above[w] = lane < 31 ? t : 0u;
   }
-  unsigned acc[W];
+  // A row can only move if some row above it is adjacent to its own column (the last step of the
+  // alternating cycle back into it): rows without such a neighbour are dropped here, which spares
+  // them a search that would reach nobody.
+  unsigned acc[W], entered[W];
 #pragma unroll
-  for (int w = 0; w < W; ++w) acc[w] = 0u;
+  for (int w = 0; w < W; ++w) acc[w] = entered[w] = 0u;
 #pragma unroll
   for (int ss = 0; ss < CPL; ++ss) {
     const int s = CPL - 1 - ss;   // from the lane's highest column down, growing gt as we go
     if (M.mr[s] >= 0) {
+      unsigned higher = 0u;
 #pragma unroll
-      for (int w = 0; w < W; ++w) acc[w] |= C[s][w] & above[w] & ~ge_word(M.mr[s], w);
+      for (int w = 0; w < W; ++w) {
+        const unsigned ge = ge_word(M.mr[s], w);
+        acc[w] |= C[s][w] & above[w] & ~ge;
+        higher |= C[s][w] & ge & ~M.word(s, w);
+      }
+      if (higher != 0u) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) entered[w] |= M.word(s, w);
+      }
     }
     M.add_to(above, s);
   }
 #pragma unroll
-  for (int w = 0; w < W; ++w) cand[w] = __reduce_or_sync(FULL, acc[w]);
+  for (int w = 0; w < W; ++w) cand[w] = __reduce_or_sync(FULL, acc[w]) & __reduce_or_sync(FULL, entered[w]);
 }
 
 // Memo carried from one call to the next when the graph only loses edges between calls
