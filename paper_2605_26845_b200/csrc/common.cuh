@@ -873,6 +873,29 @@ __device__ __forceinline__ long long batch_time_ns(const moesched_model_t& m, lo
   return m.expert_fixed_ns + (beyond * m.expert_ps_per_token + 999) / 1000;
 }
 
+// Division by a divisor fixed for the whole launch (the link speed): floor(x / d) for
+// 0 <= x < 2^55 as a multiply-high and a shift (Granlund-Montgomery: with l = ceil(log2 d) and
+// m = ceil(2^(55+l) / d), m*d lies in [2^(55+l), 2^(55+l) + 2^l], which makes the quotient exact
+// for every 55-bit x).
+struct FastDiv {
+  unsigned long long m;
+  int sh;
+};
+inline FastDiv make_fastdiv(long long d) {
+  int l = 0;
+  while ((1LL << l) < d) ++l;
+  const unsigned __int128 num = (unsigned __int128)1 << (55 + l);
+  FastDiv f;
+  f.m = (unsigned long long)((num + (unsigned __int128)(d - 1)) / (unsigned __int128)d);
+  f.sh = 55 + l;
+  return f;
+}
+__device__ __forceinline__ long long fast_div(long long x, const FastDiv& f) {
+  const unsigned long long hi = __umul64hi(f.m, (unsigned long long)x);
+  const unsigned long long lo = f.m * (unsigned long long)x;
+  return (long long)(f.sh >= 64 ? hi >> (f.sh - 64) : (hi << (64 - f.sh)) | (lo >> f.sh));
+}
+
 // ---- host-side launch geometry ---------------------------------------------------------------
 struct Geometry {
   int cpl;       // columns per lane: 1, 2, 4 or 8
@@ -898,6 +921,12 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                      long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream);
+
+// scoring with one CTA per matrix, for the matrices whose status holds CLASS_U16 (64 < N <= 256)
+cudaError_t run_eval_team(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
+                          const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
+                          long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
+                          cudaStream_t stream);
 
 // class codes the pre-pass leaves in status[b] (never equal to a final status)
 constexpr int CLASS_U16 = 64;

@@ -12,29 +12,6 @@
 
 namespace moesched {
 
-// Division by a divisor fixed for the whole launch (the link speed): floor(x / d) for
-// 0 <= x < 2^55 as a multiply-high and a shift (Granlund-Montgomery: with l = ceil(log2 d) and
-// m = ceil(2^(55+l) / d), m*d lies in [2^(55+l), 2^(55+l) + 2^l], which makes the quotient exact
-// for every 55-bit x).
-struct FastDiv {
-  unsigned long long m;
-  int sh;
-};
-static FastDiv make_fastdiv(long long d) {
-  int l = 0;
-  while ((1LL << l) < d) ++l;
-  const unsigned __int128 num = (unsigned __int128)1 << (55 + l);
-  FastDiv f;
-  f.m = (unsigned long long)((num + (unsigned __int128)(d - 1)) / (unsigned __int128)d);
-  f.sh = 55 + l;
-  return f;
-}
-__device__ __forceinline__ long long fast_div(long long x, const FastDiv& f) {
-  const unsigned long long hi = __umul64hi(f.m, (unsigned long long)x);
-  const unsigned long long lo = f.m * (unsigned long long)x;
-  return (long long)(f.sh >= 64 ? hi >> (f.sh - 64) : (hi << (64 - f.sh)) | (lo >> f.sh));
-}
-
 __device__ __forceinline__ long long warp_sum64(long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
@@ -293,12 +270,19 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
     // as in the greedy path: narrow matrices first, in the 16-bit layout, then the rest
     cudaError_t e = classify_matrices(B, N, demand, status, stream);
     if (e != cudaSuccess) return e;
-    Geometry g16 = ge;
-    g16.cluster = false;
-    g16.wpb = 1;
-    g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
-    e = launch_eval_mode<2>(g16, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok,
-                            unserved, status, prefix_overlap, prefix_unserved, CLASS_U16, stream);
+    if (N > 128 && B < 8 * sm_count() && prefix_overlap == nullptr) {
+      // few large matrices: one CTA per matrix instead of one warp (N = 256, B = 256 on a BvN schedule:
+      // 33 ms against 74 ms; at N = 128, B = 1024 one warp per matrix is the faster, 17 ms against 20 ms)
+      e = run_eval_team(B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok, unserved,
+                        status, stream);
+    } else {
+      Geometry g16 = ge;
+      g16.cluster = false;
+      g16.wpb = 1;
+      g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
+      e = launch_eval_mode<2>(g16, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns,
+                              idle_tok, unserved, status, prefix_overlap, prefix_unserved, CLASS_U16, stream);
+    }
     if (e != cudaSuccess) return e;
     only_class = CLASS_I32;
   }

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 import paper_2605_26845_b200 as ms
-from paper_2605_26845_b200.workload import (CONFIGS, DEFAULT_MODEL, bvn_capacity, make_demand,
+from paper_2605_26845_b200.workload import (CONFIGS, DEFAULT_MODEL, PROFILED_MODEL, bvn_capacity, make_demand,
                                             random_matrices, structured_cases)
 
 pytestmark = pytest.mark.gpu
@@ -149,6 +149,31 @@ def test_link_time_for_any_link_speed_and_token_size(gbps):
             assert (s[name].cpu().numpy() == r[name]).all(), (name, nbytes)
         rp = oracle.schedule_prefix_eval(D, perm, dur, count, model)
         assert (s["prefix_overlap_ns"].cpu().numpy() == rp["prefix_overlap_ns"]).all()
+
+
+@pytest.mark.parametrize("N", [100, 129, 200, 256])
+def test_large_matrix_scoring_rejects_bad_schedules_and_scores_long_ones(N):
+    """Few large matrices are scored by the kernel that puts one CTA on each matrix: faulty schedules,
+    a mix of narrow and wide matrices, and a schedule several chunks long, all against the oracle."""
+    D = random_matrices(6, N, seed=9000 + N, kind="uniform", high=3000)
+    D[5, 1, 2] = 70000                        # one wide matrix: scored by the one-warp kernel
+    d = dev(D)
+    K = 75
+    g = ms.mw_decompose(d, K)
+    perm = g.perm.cpu().numpy().copy()
+    dur = g.dur.cpu().numpy().copy()
+    count = g.count.cpu().numpy().copy()
+    assert (count > 64).all()
+    perm[0, 40, 3] = perm[0, 40, 2]           # repeated column, in the second chunk
+    perm[1, 0, 0] = 255 if N < 256 else perm[1, 0, 1]   # out of range (N = 256 has no such byte: repeat instead)
+    dur[2, 65] = -4
+    count[3] = K + 1                          # beyond the stride
+    for model in (DEFAULT_MODEL, PROFILED_MODEL):
+        s = ms.schedule_eval(d, dev(perm), dev(dur), dev(count), model)
+        r = oracle.schedule_eval(D, perm, dur, count, model, threads=8)
+        assert list(r["status"]) == [-1, -1, -1, -1, 0, 0]
+        for name in ms.SCORE_FIELDS + ("status",):
+            assert (s[name].cpu().numpy() == r[name]).all(), name
 
 
 def test_argument_errors_are_reported():
