@@ -97,6 +97,31 @@ __device__ __forceinline__ void put(T (&a)[C], int s, T v) {
 __device__ __forceinline__ unsigned onehot_word(int idx, int w) {
   return (idx >> 5) == w ? 1u << (idx & 31) : 0u;
 }
+// The one-hot mask of idx (empty for idx < 0) and the set {t, t+1, ...} as whole masks. With two
+// words (33..64 rows, the headline size) a 64-bit shift does both words at once.
+template <int W>
+__device__ __forceinline__ void onehot_mask(int idx, unsigned (&m)[W]) {
+  if constexpr (W == 2) {
+    const unsigned long long b = idx >= 0 ? 1ull << idx : 0ull;
+    m[0] = (unsigned)b;
+    m[1] = (unsigned)(b >> 32);
+  } else {
+#pragma unroll
+    for (int w = 0; w < W; ++w) m[w] = onehot_word(idx, w);
+  }
+}
+template <int W>
+__device__ __forceinline__ void ge_mask(int t, unsigned (&m)[W]) {
+  if constexpr (W == 2) {
+    const unsigned long long b = t >= 64 ? 0ull : (~0ull << (t > 0 ? t : 0));
+    m[0] = (unsigned)b;
+    m[1] = (unsigned)(b >> 32);
+  } else {
+#pragma unroll
+    for (int w = 0; w < W; ++w) m[w] = ge_word(t, w);
+  }
+}
+
 template <int W>
 __device__ __forceinline__ bool intersects(const unsigned (&a)[W], const unsigned (&b)[W]) {
   unsigned o = 0u;
@@ -131,13 +156,15 @@ struct Match {
   }
   // slot chosen at run time
   __device__ __forceinline__ void assign(int slot, int row) {
+    unsigned rowmask[CPL];
+    if constexpr (CACHED) onehot_mask<CPL>(row, rowmask);
 #pragma unroll
     for (int s = 0; s < CPL; ++s) {
       const bool me = s == slot;
       mr[s] = me ? row : mr[s];
       if constexpr (CACHED) {
 #pragma unroll
-        for (int w = 0; w < W; ++w) oh[s][w] = me ? onehot_word(row, w) : oh[s][w];
+        for (int w = 0; w < W; ++w) oh[s][w] = me ? rowmask[w] : oh[s][w];
       }
     }
   }
@@ -510,10 +537,11 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
   for (int ss = 0; ss < CPL; ++ss) {
     const int s = CPL - 1 - ss;   // from the lane's highest column down, growing gt as we go
     if (M.mr[s] >= 0) {
-      unsigned higher = 0u;
+      unsigned higher = 0u, gem[W];
+      ge_mask<W>(M.mr[s], gem);
 #pragma unroll
       for (int w = 0; w < W; ++w) {
-        const unsigned ge = ge_word(M.mr[s], w);
+        const unsigned ge = gem[w];
         acc[w] |= C[s][w] & above[w] & ~ge;
         higher |= C[s][w] & ge & ~M.word(s, w);
       }
@@ -641,11 +669,16 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
   // not covered by a record that still holds. Rebuilt only after a rotation; otherwise the row just
   // searched is simply struck off.
   unsigned todo[W];
+  {
+    unsigned lo[W], hi[W];
+    ge_mask<W>(start, lo);
+    ge_mask<W>(last + 1, hi);
 #pragma unroll
-  for (int w = 0; w < W; ++w) {
-    unsigned need = cand[w] & ge_word(start, w) & ~ge_word(last + 1, w);
-    if constexpr (MEMO) need &= ~memo.known[w];
-    todo[w] = need;
+    for (int w = 0; w < W; ++w) {
+      unsigned need = cand[w] & lo[w] & ~hi[w];
+      if constexpr (MEMO) need &= ~memo.known[w];
+      todo[w] = need;
+    }
   }
   for (int guard = 0; guard < N; ++guard) {
     const int i = lowest_bit<W>(todo);
@@ -725,10 +758,10 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       // walk towards row i: each row takes the column of its successor on the cycle
       while (lvl > 0) {
         unsigned Hm[W], cmask[W];
+        onehot_mask<W>(cur, cmask);
 #pragma unroll
         for (int w = 0; w < W; ++w) {
           Hm[w] = hist[(lvl - 1) * W + w];
-          cmask[w] = onehot_word(cur, w);
           moved[w] |= cmask[w];
         }
         int ms = -1;
@@ -762,9 +795,12 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         for (int w = 0; w < W; ++w) memo.known[w] &= ~hit[w];
       }
       candidate_rows<CPL>(lane, C, M, cand);
+      unsigned lo[W], hi[W];
+      ge_mask<W>(i + 1, lo);
+      ge_mask<W>(last + 1, hi);
 #pragma unroll
       for (int w = 0; w < W; ++w) {
-        unsigned need = cand[w] & ge_word(i + 1, w) & ~ge_word(last + 1, w);
+        unsigned need = cand[w] & lo[w] & ~hi[w];
         if constexpr (MEMO) need &= ~memo.known[w];
         todo[w] = need;
       }
@@ -792,8 +828,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   set_bit<W>(F, f);
   int t = f;
   unsigned at_or_above[W];   // rows >= t
-#pragma unroll
-  for (int w = 0; w < W; ++w) at_or_above[w] = ge_word(t, w);
+  ge_mask<W>(t, at_or_above);
   unsigned visited = 0u;
   int par[CPL];
 #pragma unroll
@@ -839,8 +874,7 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
       const int r = highest_bit<W>(P);   // admit the highest waiting row, and only that one
       if (r < 0) return false;
       t = r;
-#pragma unroll
-      for (int w = 0; w < W; ++w) at_or_above[w] = ge_word(t, w);
+      ge_mask<W>(t, at_or_above);
       clear_bit<W>(P, r);
       set_bit<W>(F, r);
     }
