@@ -25,8 +25,13 @@ enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL =
 // Bit access with a run-time index is written as arithmetic over ALL words (never as
 // "touch word k if idx/32 == k"), so that the compiler cannot turn it into an indexed
 // access that would push the register array into local memory.
+// (Two-word masks take a 64-bit path: one wide shift instead of per-word selects.)
+__device__ __forceinline__ unsigned long long as64(const unsigned (&m)[2]) {
+  return ((unsigned long long)m[1] << 32) | m[0];
+}
 template <int W>
 __device__ __forceinline__ bool test_bit(const unsigned (&m)[W], int idx) {
+  if constexpr (W == 2) return ((as64(m) >> idx) & 1ull) != 0ull;
   const unsigned bit = 1u << (idx & 31);
   const int wi = idx >> 5;
   unsigned hit = 0u;
@@ -36,6 +41,12 @@ __device__ __forceinline__ bool test_bit(const unsigned (&m)[W], int idx) {
 }
 template <int W>
 __device__ __forceinline__ void set_bit(unsigned (&m)[W], int idx) {
+  if constexpr (W == 2) {
+    const unsigned long long b = 1ull << idx;
+    m[0] |= (unsigned)b;
+    m[1] |= (unsigned)(b >> 32);
+    return;
+  }
   const unsigned bit = 1u << (idx & 31);
   const int wi = idx >> 5;
 #pragma unroll
@@ -43,6 +54,12 @@ __device__ __forceinline__ void set_bit(unsigned (&m)[W], int idx) {
 }
 template <int W>
 __device__ __forceinline__ void clear_bit(unsigned (&m)[W], int idx) {
+  if constexpr (W == 2) {
+    const unsigned long long b = 1ull << idx;
+    m[0] &= ~(unsigned)b;
+    m[1] &= ~(unsigned)(b >> 32);
+    return;
+  }
   const unsigned bit = 1u << (idx & 31);
   const int wi = idx >> 5;
 #pragma unroll
