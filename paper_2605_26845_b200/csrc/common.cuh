@@ -537,10 +537,8 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
   for (int w = 0; w < W; ++w) {
     unsigned v = own[w];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned t = __shfl_down_sync(FULL, v, o);
-      if (lane + o < 32) v |= t;
-    }
+    // (a lane whose source would lie beyond lane 31 gets its own value back: harmless in an OR)
+    for (int o = 1; o < 32; o <<= 1) v |= __shfl_down_sync(FULL, v, o);
     const unsigned t = __shfl_down_sync(FULL, v, 1);
     above[w] = lane < 31 ? t : 0u;
   }

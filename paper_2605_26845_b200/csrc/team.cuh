@@ -125,10 +125,8 @@ __device__ __forceinline__ bool team_is_candidate(TeamShared<NW>& sh, int t, int
 #pragma unroll
   for (int w = 0; w < W; ++w) {
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned u = __shfl_down_sync(FULL, v[w], o);
-      if (lane + o < 32) v[w] |= u;
-    }
+    // (a lane whose source would lie beyond lane 31 gets its own value back: harmless in an OR)
+    for (int o = 1; o < 32; o <<= 1) v[w] |= __shfl_down_sync(FULL, v[w], o);
   }
   unsigned above[W];
 #pragma unroll
