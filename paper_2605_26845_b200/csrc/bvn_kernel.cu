@@ -163,11 +163,18 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 
       // coefficient = smallest matched entry; subtract it along the matching
       int val[CPL], cmin = INF32;
+      int* cell[CPL];   // the lane's matched entries
 #pragma unroll
       for (int s = 0; s < CPL; ++s) {
         const int c = lane * CPL + s;
         val[s] = INF32;
-        if (c < N) { val[s] = A.row(M.mr[s])[c]; cmin = min(cmin, val[s]); }
+        cell[s] = nullptr;
+        if (c < N) {
+          // with the working copy in global memory every row is "near": no split to test
+          cell[s] = (MODE == 2 ? A.near_ + (size_t)M.mr[s] * A.S : A.row(M.mr[s])) + c;
+          val[s] = *cell[s];
+          cmin = min(cmin, val[s]);
+        }
       }
       cmin = __reduce_min_sync(FULL, cmin);
       lo_changed = N;
@@ -181,7 +188,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
         const int c = lane * CPL + s;
         if (c < N) {
           const int nv = val[s] - cmin;
-          A.row(M.mr[s])[c] = nv;
+          *cell[s] = nv;
           if (nv == 0) {
 #pragma unroll
             for (int w = 0; w < W; ++w) C[s][w] &= ~M.word(s, w);

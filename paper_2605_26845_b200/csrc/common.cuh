@@ -659,6 +659,28 @@ __device__ __forceinline__ void record_search(int lane, int i, const unsigned (&
   if constexpr (!CanonMemo<W>::IN_REGS) __syncwarp();
 }
 
+// One row set of the search history (W words at hist + level * W): written by one lane, with a
+// single 8-byte store when the set has two words.
+template <int W>
+__device__ __forceinline__ void hist_store(unsigned* hist, int level, const unsigned (&F)[W], int lane) {
+  if constexpr (W == 2) {
+    if (lane == 0) *reinterpret_cast<uint2*>(hist + level * 2) = make_uint2(F[0], F[1]);
+  } else {
+    if (lane < W) hist[level * W + lane] = pick<W>(F, lane);
+  }
+}
+template <int W>
+__device__ __forceinline__ void hist_load(const unsigned* hist, int level, unsigned (&H)[W]) {
+  if constexpr (W == 2) {
+    const uint2 v = *reinterpret_cast<const uint2*>(hist + level * 2);
+    H[0] = v.x;
+    H[1] = v.y;
+  } else {
+#pragma unroll
+    for (int w = 0; w < W; ++w) H[w] = hist[level * W + w];
+  }
+}
+
 template <int CPL, bool MEMO>
 __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int last,
                                              const unsigned (&C)[CPL][CPL], Match<CPL>& M, short* x,
@@ -710,14 +732,14 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         const unsigned lowbit = todo[w] & (0u - todo[w]);
         const bool here = below && todo[w] != 0u;
         imask[w] = here ? lowbit : 0u;
-        alive[w] = here ? (0u - lowbit) : (below ? 0u : 0xffffffffu);
+        alive[w] = here ? (0u - lowbit) & ~lowbit : (below ? 0u : 0xffffffffu);   // rows above i
         below = below && todo[w] == 0u;
         todo[w] &= ~imask[w];
         anc[w] = F[w] = imask[w];
       }
     }
     int level = 0;
-    if (lane < W) hist[lane] = pick<W>(F, lane);
+    hist_store<W>(hist, 0, F, lane);
     for (int it = 0; it < N; ++it) {
       unsigned acc[W];
 #pragma unroll
@@ -732,7 +754,8 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       bool grew = false;
 #pragma unroll
       for (int w = 0; w < W; ++w) {
-        unsigned a = __reduce_or_sync(FULL, acc[w]) & alive[w] & ~anc[w];
+        const unsigned a = __reduce_or_sync(FULL, acc[w]) & alive[w];   // alive: rows >= i not reached yet
+        alive[w] &= ~a;
         anc[w] |= a;
         F[w] = a;
         grew |= a != 0u;
@@ -740,7 +763,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       work[WK_LEVEL]++;
       if (!grew) break;
       ++level;
-      if (lane < W) hist[level * W + lane] = pick<W>(F, lane);
+      hist_store<W>(hist, level, F, lane);
     }
     __syncwarp();
     // lowest column row i may take (its own column always qualifies)
@@ -774,11 +797,9 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       while (lvl > 0) {
         unsigned Hm[W], cmask[W];
         onehot_mask<W>(cur, cmask);
+        hist_load<W>(hist, lvl - 1, Hm);
 #pragma unroll
-        for (int w = 0; w < W; ++w) {
-          Hm[w] = hist[(lvl - 1) * W + w];
-          moved[w] |= cmask[w];
-        }
+        for (int w = 0; w < W; ++w) moved[w] |= cmask[w];
         int ms = -1;
 #pragma unroll
         for (int ss = 0; ss < CPL; ++ss) {
