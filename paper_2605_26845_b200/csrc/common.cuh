@@ -539,8 +539,9 @@ __device__ __forceinline__ void candidate_rows(int lane, const unsigned (&C)[CPL
 #pragma unroll
     // (a lane whose source would lie beyond lane 31 gets its own value back: harmless in an OR)
     for (int o = 1; o < 32; o <<= 1) v |= __shfl_down_sync(FULL, v, o);
-    const unsigned t = __shfl_down_sync(FULL, v, 1);
-    above[w] = lane < 31 ? t : 0u;
+    // v now covers this lane and all higher ones; every row is matched to one column only, so
+    // taking the lane's own rows out leaves exactly the rows of the higher lanes
+    above[w] = v & ~own[w];
   }
   // A row can only move if some row above it is adjacent to its own column (the last step of the
   // alternating cycle back into it): rows without such a neighbour are dropped here, which spares
