@@ -131,8 +131,9 @@ __device__ __forceinline__ bool team_is_candidate(TeamShared<NW>& sh, int t, int
   unsigned above[W];
 #pragma unroll
   for (int w = 0; w < W; ++w) {
-    const unsigned u = __shfl_down_sync(FULL, v[w], 1);
-    above[w] = lane < 31 ? u : 0u;
+    // v covers this row and all higher rows of the warp; a column is matched to one row only, so
+    // taking the row's own column out leaves exactly the columns of the higher rows
+    above[w] = v[w] & ~(in ? onehot_word(m.my_x, w) : 0u);
     const unsigned total = __shfl_sync(FULL, v[w], 0);
     if (lane == w) sh.tot[warp * W + w] = total;
   }
