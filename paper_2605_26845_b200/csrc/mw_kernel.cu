@@ -160,11 +160,10 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
       const int i = __shfl_sync(FULL, st.M.row_of(sl), L);
       work[WK_SCAN]++;
       if (i < 0) { jfin = L * CPL + sl; break; }
-      const int vj = __shfl_sync(FULL, pick<CPL>(st.v, sl), L);
       RowVec<CPL> rv;
       if (lane_in) rv = load_cols<CPL>(R.row(i), lane);
-      const int rij = __shfl_sync(FULL, pick<CPL>(rv.v, sl), L);
-      const int h = -rij - vj - mu;
+      // the owner of the settled column forms h from its own entry and dual: one broadcast instead of two
+      const int h = __shfl_sync(FULL, -pick<CPL>(rv.v, sl) - pick<CPL>(st.v, sl) - mu, L);
 #pragma unroll
       for (int s = 0; s < CPL; ++s) {
         int nd = -rv.v[s] - st.v[s] - h;
