@@ -103,6 +103,9 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   const uint8_t* pb = perm + (size_t)b * k_stride * N;
   const int32_t* db = dur + (size_t)b * k_stride;
 
+  unsigned allcols[W];   // the set of all N columns
+#pragma unroll
+  for (int w = 0; w < W; ++w) allcols[w] = ~ge_word(N, w);
   if (!bad) {
     // one aligned word holds the lane's CPL destinations when rows of the schedule are CPL-aligned
     const bool packed_ok = (N % CPL == 0) && ((reinterpret_cast<uintptr_t>(pb) & (CPL - 1)) == 0);
@@ -153,10 +156,11 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
               }
             }
           }
-          int seen = 0;
+          // N destinations, none out of range: a permutation iff every column 0..N-1 is hit
+          unsigned missing = 0u;
 #pragma unroll
-          for (int w = 0; w < W; ++w) seen += __popc(__reduce_or_sync(FULL, cols[w]));
-          if (__any_sync(FULL, oob) || seen != N) {
+          for (int w = 0; w < W; ++w) missing |= ~__reduce_or_sync(FULL, cols[w]) & allcols[w];
+          if (__any_sync(FULL, oob) || missing != 0u) {
             bad = 1;
           } else {
             g = __reduce_max_sync(FULL, g);
