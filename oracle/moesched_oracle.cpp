@@ -393,8 +393,8 @@ struct Model {
 
 i64 cdiv(i64 x, i64 y) { return (x + y - 1) / y; }
 
-// Time of one expert batch of g tokens on the busiest rank [Sec. 2.2 "Compute time is not
-// strictly linear", Fig. 1]: nothing to do costs nothing; up to the knee the fixed overhead
+// Time of one expert batch of g tokens on the busiest rank [Sec. 2.2, the paragraph on the
+// shape of the compute-time curve; Fig. 1]: nothing to do costs nothing; up to the knee the fixed overhead
 // dominates (flat); beyond it the time grows linearly. knee = 0 gives the affine model.
 i64 batch_time(const Model& m, i64 g) {
   if (g <= 0) return 0;
@@ -561,8 +561,8 @@ int oracle_schedule_prefix_eval(int B, int N, const int32_t* demand, int k_strid
   return 0;
 }
 
-// Idealised congestion-free all-to-all [Sec. 4.1 "Comparisons": "the theoretical completion
-// time for a given communication matrix"]: every port sends and receives at line rate, so the
+// Idealised congestion-free all-to-all [Sec. 4.1 "Comparisons": the best completion time any
+// fabric could reach for the matrix]: every port sends and receives at line rate, so the
 // exchange lasts as long as the busiest port (largest row or column sum); like the sequential
 // baseline it runs dispatch, compute and combine to completion one after the other, with all
 // tokens of a rank in one batch and no circuit reconfiguration.
@@ -595,9 +595,12 @@ int oracle_ideal_a2a(int B, int N, const int32_t* demand, const int64_t* model, 
 // Sinkhorn-Knopp scaling [Sec. 3.1: the preprocessing the paper names for making a demand matrix
 // doubly stochastic before the Birkhoff-von Neumann decomposition]. The paper gives no constants,
 // so the steps are spelled out here: X = D + smooth (smooth > 0 gives every pair a little mass, so
-// that zero rows and columns can be scaled at all); one sweep multiplies every row by the
-// reciprocal of its sum, then every column by the reciprocal of its sum (the usual statement of
-// the iteration: u = 1 / (X v), v = 1 / (X^T u)); `iters` sweeps. All arithmetic is IEEE double,
+// that zero rows and columns can be scaled at all); one sweep normalises the rows and then the
+// columns, which is the method's own definition: every entry is DIVIDED by the sum of its row,
+// then every entry by the sum of its column; `iters` sweeps. Dividing (rather than multiplying by
+// a rounded reciprocal) is the plain reading of "normalise", and it keeps what a normalisation
+// promises: an entry that is its whole row or column becomes exactly 1, and a constant matrix m*J
+// becomes exactly J/N whenever 1/N is representable, for any m. All arithmetic is IEEE double,
 // sums run left to right (rows) and top to bottom (columns), one rounding per operation.
 //   scaled   = the matrix after the last sweep (column sums 1 up to rounding, row sums 1 + row_err);
 //   fixed    = round-half-up(scaled * 2^scale_bits): the integer matrix handed to the exact
@@ -629,15 +632,13 @@ int oracle_sinkhorn_scale(int B, int N, const int32_t* demand, int iters, double
         double r = 0.0;
         for (int j = 0; j < N; ++j) r = r + S[i * N + j];
         if (!(r > 0.0)) bad = true;
-        const double u = 1.0 / r;
-        for (int j = 0; j < N; ++j) S[i * N + j] = S[i * N + j] * u;
+        for (int j = 0; j < N; ++j) S[i * N + j] = S[i * N + j] / r;
       }
       for (int j = 0; j < N; ++j) {
         double c = 0.0;
         for (int i = 0; i < N; ++i) c = c + S[i * N + j];
         if (!(c > 0.0)) bad = true;
-        const double v = 1.0 / c;
-        for (int i = 0; i < N; ++i) S[i * N + j] = S[i * N + j] * v;
+        for (int i = 0; i < N; ++i) S[i * N + j] = S[i * N + j] / c;
       }
     }
     if (bad) {

@@ -64,14 +64,20 @@ def test_against_a_vectorised_statement_and_sweep_by_sweep_error():
 
 def test_balanced_inputs_and_power_of_two_invariance():
     N = 8                                                # 1/8 is exact in binary floating point
-    J = np.full((1, N, N), 8, np.int32)
-    r = oracle.sinkhorn_scale(J, 1, 0.0, 20)
-    assert (r["scaled"] == 1.0 / N).all() and r["row_err"][0] < 1e-15
-    P = np.zeros((1, N, N), np.int32)
-    P[0, np.arange(N), np.roll(np.arange(N), 2)] = 16
-    r = oracle.sinkhorn_scale(P, 3, 0.0, 20)
-    assert (r["scaled"][0] == (P[0] > 0)).all()
-    assert (r["fixed"][0] == (P[0] > 0) * 2**20).all() and r["stretch"][0] == 16.0
+    # a normalisation divides: m * J becomes exactly J / N for ANY m, not only for powers of two
+    # (m / (m N) is correctly rounded to 1 / N; m times a rounded 1 / (m N) would not be)
+    for m in (7, 8, 12, 1000, 4093):
+        J = np.full((1, N, N), m, np.int32)
+        r = oracle.sinkhorn_scale(J, 1, 0.0, 20)
+        assert (r["scaled"] == 1.0 / N).all() and r["row_err"][0] == 0.0, m
+        assert (r["fixed"] == 2**20 // N).all() and r["stretch"][0] == float(m * N)
+    # an entry that is its whole row and column becomes exactly 1 whatever its value
+    for m in (12, 16, 4093):
+        P = np.zeros((1, N, N), np.int32)
+        P[0, np.arange(N), np.roll(np.arange(N), 2)] = m
+        r = oracle.sinkhorn_scale(P, 3, 0.0, 20)
+        assert (r["scaled"][0] == (P[0] > 0)).all()
+        assert (r["fixed"][0] == (P[0] > 0) * 2**20).all() and r["stretch"][0] == float(m)
     D = random_matrices(2, 9, seed=3, kind="uniform", high=100)
     a = oracle.sinkhorn_scale(D, 7, 0.5, 16)
     b = oracle.sinkhorn_scale(D * 4, 7, 2.0, 16)        # scaling by a power of two is exact in binary floating point
