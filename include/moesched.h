@@ -90,9 +90,9 @@ typedef struct moesched_model {
 } moesched_model_t;
 
 /*
- * Greedy max-weight decomposition (paper Sec. 3.2: "repeatedly extracts the
- * maximum-weight perfect matching from the residual matrix and subtracts the
- * selected matching until all entries become zero").
+ * Greedy max-weight decomposition (paper Sec. 3.2): a maximum-weight perfect
+ * matching of what is left of the matrix is taken out again and again until
+ * nothing is left, or until the budget k_max is used up.
  *
  * Per matrix: R <- D; while k < k_max and R != 0: pi_k <- lexicographically
  * smallest permutation maximising sum_i R[i][pi(i)] (zero entries are ordinary
@@ -163,13 +163,19 @@ int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uin
  * (B * N * roundup(N, 8) * 4); 0 for sizes out of range. */
 size_t moesched_bvn_scratch_bytes(int B, int N);
 
+/* Device working memory, in bytes, that a pass of the whole path over B matrices of size N can
+ * use beyond its inputs and outputs, whatever the budget k_max: the greedy decomposition and the
+ * scoring keep their working state in shared memory and need none, so this is the scratch of the
+ * Birkhoff-von Neumann decomposition (moesched_bvn_scratch_bytes). 0 for sizes out of range
+ * (B < 0, N outside 1..256, k_max < 1). */
+size_t moesched_workspace_bytes(int B, int N, int k_max);
+
 /*
- * Score a schedule (paper Sec. 4.1: a matching completes after its largest
- * transfer; "after the dispatch phase of the i-th matching completes, expert
- * computation begins immediately while communication for the (i+1)-th matching
- * progresses"; Sec. 3.3: dispatch, compute and combine form a three-machine
- * flow shop; the "no overlap" panels of Fig. 3 / Fig. 4 run every phase to
- * completion).
+ * Score a schedule (paper Sec. 4.1 "Execution time": a matching completes after
+ * its largest transfer, and the experts start on a matching as soon as its
+ * dispatch is done, while the next matching is already being sent; Sec. 3.3:
+ * dispatch, compute and combine form a three-machine flow shop; the panels of
+ * Fig. 3 / Fig. 4 without overlap run every phase to completion).
  *
  * Per matrix, replaying matchings k = 0 .. count-1 against D:
  *   served_i = min(dur_k, Dres[i][pi_k(i)]); Dres -= served  (real tokens first)
@@ -219,9 +225,9 @@ int moesched_schedule_prefix_eval(int B, int N, const int32_t* d_demand, int k_s
                                   int64_t* d_prefix_unserved_tokens, void* stream);
 
 /*
- * Idealised congestion-free all-to-all (paper Sec. 4.1 "Comparisons": "the theoretical
- * completion time for a given communication matrix"), the yardstick the decomposed
- * schedules are compared with. Every port sends and receives at line rate, so one exchange
+ * Idealised congestion-free all-to-all (paper Sec. 4.1 "Comparisons": the best completion time
+ * any fabric could reach for the matrix), the yardstick the decomposed schedules are compared
+ * with. Every port sends and receives at line rate, so one exchange
  * lasts as long as its busiest port; dispatch, expert compute (all tokens of a rank in one
  * batch) and combine run to completion one after the other; no circuit is reconfigured.
  *   port_b  = max(largest row sum, largest column sum) of matrix b
@@ -239,17 +245,16 @@ int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_mod
 
 /*
  * Sinkhorn-Knopp scaling: the preprocessing the paper names for the Birkhoff-von Neumann
- * decomposition (Sec. 3.1: "a preprocessing step such as Sinkhorn-Knopp normalization is
- * required before decomposition can be applied"; it "redistributes communication mass across
- * rows and columns" and so "introduces idle capacity that does not correspond to the original
- * routing demand"). moesched_bvn_decompose pads instead; this entry point gives the paper's
+ * decomposition (Sec. 3.1: demand matrices are not doubly stochastic, so they are normalised
+ * first; the normalisation moves mass between rows and columns and thereby adds capacity that
+ * no routed token asked for). moesched_bvn_decompose pads instead; this entry point gives the paper's
  * multiplicative route: scale here, then decompose d_fixed with moesched_bvn_decompose, turn
  * its coefficients into token counts with moesched_sinkhorn_durations, and score the result
  * against the ORIGINAL demand with moesched_schedule_eval.
  *
- * The paper fixes no constants; the steps are: X = D + smooth; one sweep multiplies every row of
- * X by the reciprocal of its sum and then every column by the reciprocal of its sum; `iters`
- * sweeps. IEEE double arithmetic, row sums accumulated left to right and column sums top to
+ * The paper fixes no constants; the steps are: X = D + smooth; one sweep divides every entry of
+ * X by the sum of its row and then every entry by the sum of its column; `iters` sweeps. IEEE
+ * double arithmetic, row sums accumulated left to right and column sums top to
  * bottom, one rounding per operation -- the result is therefore reproducible bit for bit.
  *   d_scaled[b]  = X after the last sweep (column sums 1 up to rounding)
  *   d_row_err[b] = max_i |sum_j scaled[b][i][j] - 1|, the distance from double stochasticity
@@ -329,8 +334,13 @@ long long moesched_probe_int_ops(int blocks, int iters, uint32_t* d_out, void* s
  * this library on the calling thread; 0 if none. */
 int moesched_last_cuda_error(void);
 
-/* Text for a MOESCHED_* return code or MOESCHED_ST_* status. Never NULL. */
+/* Text for a MOESCHED_* RETURN CODE of an entry point (MOESCHED_OK, _EINVAL, _ECUDA, _ETOOBIG).
+ * Never NULL. Per-matrix statuses share small numbers with the return codes and have their own
+ * function below. */
 const char* moesched_strerror(int code);
+
+/* Text for a per-matrix MOESCHED_ST_* value read from a d_status array. Never NULL. */
+const char* moesched_status_str(int status);
 
 #ifdef __cplusplus
 }

@@ -46,6 +46,8 @@ def load_library():
                                 "(there is no CPU fallback)")
         lib = ctypes.CDLL(LIB_PATH)
         lib.moesched_strerror.restype = ctypes.c_char_p
+        lib.moesched_status_str.restype = ctypes.c_char_p
+        lib.moesched_workspace_bytes.restype = ctypes.c_size_t
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
                      "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
                      "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error"):
@@ -128,6 +130,16 @@ def mw_decompose(demand, k_max, want_residual=False, want_work=False, out=None) 
 
 def bvn_scratch_bytes(B, N) -> int:
     return int(load_library().moesched_bvn_scratch_bytes(int(B), int(N)))
+
+
+def workspace_bytes(B, N, k_max) -> int:
+    """Device working memory a pass of the whole path can use beyond its inputs and outputs."""
+    return int(load_library().moesched_workspace_bytes(int(B), int(N), int(k_max)))
+
+
+def status_str(status) -> str:
+    """Text for one per-matrix status value."""
+    return load_library().moesched_status_str(int(status)).decode()
 
 
 def bvn_decompose(demand, k_max=None, want_aug=False, want_work=False, out=None, scratch=True) -> Schedule:

@@ -79,6 +79,11 @@ size_t moesched_bvn_scratch_bytes(int B, int N) {
   return (size_t)B * N * bvn_scratch_stride(N) * sizeof(int32_t);
 }
 
+size_t moesched_workspace_bytes(int B, int N, int k_max) {
+  if (k_max < 1) return 0;
+  return moesched_bvn_scratch_bytes(B, N);
+}
+
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm, int32_t* d_coef,
                            int32_t* d_count, int32_t* d_aug, int32_t* d_scratch, int32_t* d_status,
                            int64_t* d_work, void* stream) {
@@ -191,11 +196,20 @@ int moesched_last_cuda_error(void) { return g_last_cuda_error; }
 const char* moesched_strerror(int code) {
   switch (code) {
     case MOESCHED_OK: return "ok";
-    case MOESCHED_ST_TRUNCATED: return "truncated: the matching budget ran out before the matrix did";
-    case MOESCHED_EINVAL: return "invalid argument, or (as a status) input matrix out of range";
-    case MOESCHED_ECUDA: return "a CUDA call failed, or (as a status) an internal iteration limit was hit";
+    case MOESCHED_EINVAL: return "invalid argument: null or misaligned pointer, or a size out of range";
+    case MOESCHED_ECUDA: return "a CUDA call failed (see moesched_last_cuda_error)";
     case MOESCHED_ETOOBIG: return "batch too large for the library's built-in scratch array";
-    default: return "unknown moesched code";
+    default: return "unknown moesched return code";
+  }
+}
+
+const char* moesched_status_str(int status) {
+  switch (status) {
+    case MOESCHED_ST_OK: return "ok: complete result";
+    case MOESCHED_ST_TRUNCATED: return "truncated: the matching budget ran out before the matrix did";
+    case MOESCHED_ST_BAD_INPUT: return "bad input: the matrix or schedule violates the documented range";
+    case MOESCHED_ST_INTERNAL: return "internal: an iteration limit was hit (a bug in the library)";
+    default: return "unknown moesched status";
   }
 }
 

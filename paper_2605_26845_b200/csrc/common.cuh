@@ -1,6 +1,7 @@
-// Device-side building blocks shared by the three kernels: one warp owns one
-// demand matrix, held in shared memory (for N > 128 spread over the two CTAs of
-// a thread-block cluster), and keeps the matching state in registers.
+// Device-side building blocks shared by the kernels in which one warp owns one
+// demand matrix: the matrix is held in shared memory (as int32 above 232 ranks it
+// is spread over the two CTAs of a thread-block cluster) or in a global working
+// copy, and the matching state lives in registers.
 //
 // Ownership: lane l owns columns (and rows, where a per-row value is kept in
 // registers) l*CPL .. l*CPL+CPL-1, CPL = 1, 2, 4 or 8, so that a row scan is one

@@ -1,8 +1,8 @@
 // Sinkhorn-Knopp scaling (the preprocessing paper Sec. 3.1 names for the Birkhoff-von Neumann
 // decomposition), one warp per demand matrix, IEEE double throughout.
 //
-// X = D + smooth; one sweep multiplies every row by the reciprocal of its sum, then every column
-// by the reciprocal of its sum. The sums are defined left to right (rows) and top to bottom
+// X = D + smooth; one sweep divides every entry by the sum of its row, then every entry by the sum
+// of its column (IEEE division, correctly rounded). The sums are defined left to right (rows) and top to bottom
 // (columns) with one rounding per operation, so that the result does not depend on how the work
 // is spread over lanes:
 //   * a column sum is accumulated by the lane that owns the column (column c: lane c % 32) while
@@ -25,10 +25,10 @@ namespace {
 constexpr int SK_TILE = 32 * 33;          // doubles of the tile
 constexpr int SK_WARP = SK_TILE + 256;    // plus one row sum per row
 
-// Applies the pending column scaling (entry (r, c) times col_mul of its column) if HAVE_MUL, writes
+// Applies the pending column scaling (entry (r, c) divided by col_div of its column) if HAVE_MUL, writes
 // the scaled entries back, and leaves in rsum[r] (shared memory) the sum of row r, left to right.
 template <int CPL, bool HAVE_MUL>
-__device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double* tile, const double (&col_mul)[CPL],
+__device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double* tile, const double (&col_div)[CPL],
                                               double* rsum) {
   for (int rb = 0; rb * 32 < N; ++rb) {
     double acc = 0.0;
@@ -42,7 +42,7 @@ __device__ __forceinline__ void row_sums_pass(int N, int lane, double* S, double
           if (r < N && c < N) {
             v = S[(size_t)r * N + c];
             if (HAVE_MUL) {
-              v = __dmul_rn(v, col_mul[cb]);
+              v = __ddiv_rn(v, col_div[cb]);
               S[(size_t)r * N + c] = v;
             }
           }
@@ -87,21 +87,17 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
   bad = __any_sync(FULL, bad);
   __syncwarp();
 
-  double col_mul[CPL];
+  double col_div[CPL];   // column sums of the last column pass: the division by them is still pending
 #pragma unroll
-  for (int s = 0; s < CPL; ++s) col_mul[s] = 1.0;
+  for (int s = 0; s < CPL; ++s) col_div[s] = 1.0;
   for (int it = 0; it < iters && !bad; ++it) {
-    if (it == 0) row_sums_pass<CPL, false>(N, lane, S, tile, col_mul, rsum);
-    else row_sums_pass<CPL, true>(N, lane, S, tile, col_mul, rsum);
+    if (it == 0) row_sums_pass<CPL, false>(N, lane, S, tile, col_div, rsum);
+    else row_sums_pass<CPL, true>(N, lane, S, tile, col_div, rsum);
     // a row without mass cannot be scaled
     int zero = 0;
     for (int r = lane; r < N; r += 32) zero |= !(rsum[r] > 0.0);
     if (__any_sync(FULL, zero)) { bad = 1; break; }
-    // each lane turns the sums of its rows into reciprocals
-    __syncwarp();
-    for (int r = lane; r < N; r += 32) rsum[r] = __ddiv_rn(1.0, rsum[r]);
-    __syncwarp();
-    // scale the rows and accumulate the column sums from the top
+    // divide the rows by their sums and accumulate the column sums from the top
     double csum[CPL];
 #pragma unroll
     for (int s = 0; s < CPL; ++s) csum[s] = 0.0;
@@ -111,7 +107,7 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
       for (int s = 0; s < CPL; ++s) {
         const int c = s * 32 + lane;
         if (c < N) {
-          const double v = __dmul_rn(S[(size_t)r * N + c], rv);
+          const double v = __ddiv_rn(S[(size_t)r * N + c], rv);
           S[(size_t)r * N + c] = v;
           csum[s] = __dadd_rn(csum[s], v);
         }
@@ -121,7 +117,7 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
 #pragma unroll
     for (int s = 0; s < CPL; ++s) {
       if (s * 32 + lane < N) zero |= !(csum[s] > 0.0);
-      col_mul[s] = __ddiv_rn(1.0, csum[s]);
+      col_div[s] = csum[s];
     }
     if (__any_sync(FULL, zero)) { bad = 1; break; }
     __syncwarp();
@@ -135,7 +131,7 @@ __global__ void __launch_bounds__(128) sinkhorn_kernel(int B, int N, const int32
   }
 
   // the last column scaling, the row sums of the result, the fixed-point matrix and the stretch
-  row_sums_pass<CPL, true>(N, lane, S, tile, col_mul, rsum);
+  row_sums_pass<CPL, true>(N, lane, S, tile, col_div, rsum);
   double err = 0.0;
   for (int r = lane; r < N; r += 32) err = fmax(err, fabs(__dadd_rn(rsum[r], -1.0)));
   __syncwarp();

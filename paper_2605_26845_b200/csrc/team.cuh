@@ -214,6 +214,16 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
     const int i = (int)(ikey >> 16);
     from = i + 1;
     if (t == 0) work[WK_SWEEP]++;
+    // Every search takes a fresh range of N + 2 level stamps, so that the marks of earlier searches
+    // never need clearing. Before the stamps could pass 2^31 (after some 8 million searches at
+    // N = 256; a complete worst-case decomposition can get there) all marks are wiped and the
+    // stamps start over. stamp is uniform, so every thread takes this branch or none does.
+    if (stamp > 0x7f000000) {
+      __syncthreads();
+      sh.lvl[t] = -1;
+      stamp = 0;
+      __syncthreads();
+    }
     stamp += N + 2;
     // level 0: row i itself. Its adjacency is published for the column choice (read several
     // barriers later; the previous search's readers are past the barrier above).

@@ -3,7 +3,8 @@
 The paper evaluates on routing traces of Mixtral 8x7B, Mixtral 8x22B and
 DeepSeek-MoE-16B over two prompt datasets (Sec. 4); neither the traces nor the
 datasets are available here, so token-routing matrices with the same
-character ("sparse, highly skewed, and imbalanced", Sec. 2.2) are drawn from
+character (few heavy pairs, many light or empty ones, unequal row and column
+sums: Sec. 2.2) are drawn from
 a stated recipe instead. D[b, i, j] is the number of (token, expert) selections
 that rank i sends to rank j in all-to-all b; the diagonal (tokens that stay on
 their own rank) is kept.
