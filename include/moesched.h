@@ -309,11 +309,14 @@ int moesched_sinkhorn_durations(int B, int k_stride, const int32_t* d_coef, cons
  *
  * The first call on each device looks up the array's device address (no allocation, but
  * a runtime query): make that first call with the device current and outside any stream
- * capture. All calls share the one array; it holds whatever the previous call left and is
- * fully rewritten for the rows it uses, so nothing needs clearing, but two calls that can
- * run at the same time on one GPU (different streams, threads or processes sharing a
- * context) would trample each other's working copy: serialise them. No cudaMalloc,
- * cudaFree or other allocating call is made.
+ * capture. The address is remembered per device for the life of the process; a caller that
+ * resets the device (cudaDeviceReset) afterwards must not call this entry point again,
+ * because the remembered address then points into a context that no longer exists.
+ * All calls of one process on one GPU share the one array (another process has its own copy);
+ * it holds whatever the previous call left and is fully rewritten for the rows it uses, so
+ * nothing needs clearing, but two calls that can run at the same time on one GPU (from
+ * different streams or threads of the process) would trample each other's working copy:
+ * serialise them. No cudaMalloc, cudaFree or other allocating call is made.
  */
 #define MOESCHED_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
 int moesched_bvn_decompose_static(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,

@@ -86,6 +86,50 @@ def test_team_kernel_deep_prefix(N, kw):
         assert (v.extra.cpu().numpy() == rv["aug"]).all()
 
 
+@pytest.mark.parametrize("N,kw", [(129, KINDS[2]), (256, KINDS[0])])
+def test_one_warp_kernel_above_128_ranks_in_a_large_batch(N, kw):
+    """Above 128 ranks a batch of at least eight matrices per SM keeps one warp per matrix, with the
+    working copy in global memory and the search records in shared memory; a small batch of the same
+    matrices takes the CTA-per-matrix kernel. Both against the oracle on a sample, and against each
+    other on every matrix."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    base = random_matrices(37, N, seed=8100 + N, **kw)
+    reps = -(-8 * sms // base.shape[0])
+    D = np.concatenate([base] * reps)
+    assert D.shape[0] >= 8 * sms
+    K = 24
+    wide = ms.bvn_decompose(dev(D), K, want_aug=True)
+    small = ms.bvn_decompose(dev(base), K, want_aug=True)
+    rv = oracle.bvn_decompose(base, K, threads=8)
+    assert_schedule_equal(small, rv, "coef")
+    for q in range(reps):
+        part = ms.Schedule(*(getattr(wide, f)[q * 37:(q + 1) * 37] for f in ("perm", "dur", "count", "status")))
+        assert_schedule_equal(part, rv, "coef")
+    assert (wide.extra[:37].cpu().numpy() == rv["aug"]).all()
+
+
+@pytest.mark.parametrize("N", [233, 256])
+def test_wide_entries_above_232_ranks_run_deep_on_the_cluster_path(N):
+    """Entries beyond 16 bits at N > 232 put the matrix (as int32) across the two CTAs of a cluster, for
+    the greedy decomposition and for the scoring alike: 70 matchings deep against the oracle."""
+    D = random_matrices(3, N, seed=8300 + N, kind="uniform", high=400000, zero_frac=0.5)
+    D[2] = np.minimum(D[2], 65535)                       # one narrow matrix in the same batch
+    d = dev(D)
+    K = 70
+    g = ms.mw_decompose(d, K, want_residual=True)
+    rg = oracle.mw_decompose(D, K, threads=8)
+    assert_schedule_equal(g, rg, "dur")
+    assert (g.extra.cpu().numpy() == rg["residual"]).all() and (rg["count"] == K).all()
+    for model in (DEFAULT_MODEL, PROFILED_MODEL):
+        s = ms.schedule_eval(d, g.perm, g.dur, g.count, model, prefix=True)
+        rs = oracle.schedule_eval(D, rg["perm"], rg["dur"], rg["count"], model, threads=8)
+        for name in ms.SCORE_FIELDS + ("status",):
+            assert (s[name].cpu().numpy() == rs[name]).all(), name
+        rp = oracle.schedule_prefix_eval(D, rg["perm"], rg["dur"], rg["count"], model, threads=8)
+        assert (s["prefix_overlap_ns"].cpu().numpy() == rp["prefix_overlap_ns"]).all()
+        assert (s["prefix_unserved_tokens"].cpu().numpy() == rp["prefix_unserved_tokens"]).all()
+
+
 @pytest.mark.parametrize("N", [1, 2, 5, 8, 17, 64, 100])
 def test_closed_form_cases(N):
     cases = structured_cases(N, m=7)

@@ -125,3 +125,22 @@ def test_pins_separate_plausible_mistakes():
     assert list(oracle.max_weight_perm(W2, 1)) == [1, 0, 2]
     # highest column on ties would give [1, 0]
     assert list(oracle.max_weight_perm(np.array([[3, 3], [3, 3]]), 1)) == [0, 1]
+
+
+def test_forced_assignment_agrees_at_64_ranks_on_workload_matrices():
+    """Tier 2 (forced assignment: uses optimal VALUES only, no tight graph, no alternating cycles) against
+    tier 1 at the headline size, where the big comparisons otherwise rest on tier 1 alone: the first
+    matchings of the greedy and of the Birkhoff decomposition of two matrices of configuration 3."""
+    from paper_2605_26845_b200.workload import make_demand
+    D = make_demand(3, 2)
+    K = 6
+    a = oracle.mw_decompose(D, K, tier=1, threads=2)
+    b = oracle.mw_decompose(D, K, tier=2, threads=2)
+    assert (a["count"] == K).all() and (b["count"] == K).all()
+    assert (a["perm"] == b["perm"]).all() and (a["dur"] == b["dur"]).all()
+    assert (a["residual"] == b["residual"]).all()
+    K = 8
+    a = oracle.bvn_decompose(D, K, tier=1, threads=2)
+    b = oracle.bvn_decompose(D, K, tier=2, threads=2)
+    assert (a["count"] == K).all() and (b["count"] == K).all()
+    assert (a["perm"] == b["perm"]).all() and (a["coef"] == b["coef"]).all()
