@@ -67,7 +67,7 @@ extern "C" {
 #define MOESCHED_MW_MAX_ENTRY 268435456
 
 /* Number of int64 work counters per matrix written to d_work (see below). */
-#define MOESCHED_WORK_FIELDS 8
+#define MOESCHED_WORK_FIELDS 10
 
 /* Link and compute model of the overlap pipeline (paper Sec. 4.1 "Execution
  * time"): a matching lasts as long as its largest transfer at link speed; an
@@ -113,7 +113,9 @@ typedef struct moesched_model {
  *                   tried against their best column, 3 canonicalisation
  *                   sweeps that searched, 4 search levels, 5 rotation steps,
  *                   6 matchings, 7 rows matched along tight edges before the
- *                   shortest-path phase
+ *                   shortest-path phase, 8 rows expanded by the canonicalisation
+ *                   searches (frontier pops), 9 groups of columns settled together
+ *                   (CTA-per-matrix kernel only; there 0 counts the rows relaxed)
  */
 int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                           int32_t* d_dur, int32_t* d_count, int32_t* d_residual,
@@ -153,7 +155,8 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
  *                   search levels, 1 augmenting-path steps, 2 matchings
  *                   repaired, 3 canonicalisation sweeps that searched,
  *                   4 search levels, 5 rotation steps, 6 matchings, 7 rows
- *                   skipped as unchanged prefix
+ *                   skipped as unchanged prefix, 8 rows expanded by the
+ *                   canonicalisation searches (frontier pops), 9 unused
  */
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                            int32_t* d_coef, int32_t* d_count, int32_t* d_aug, int32_t* d_scratch,

@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmoesched.so")
 
 ST_OK, ST_TRUNCATED, ST_BAD_INPUT, ST_INTERNAL = 0, 1, -1, -2
-WORK_FIELDS = 8
+WORK_FIELDS = 10
 MAX_N = 256
 
 

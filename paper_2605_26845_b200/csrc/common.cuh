@@ -19,7 +19,7 @@ namespace moesched {
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int INF32 = 0x7fffffff;
 
-enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL = 4, WK_ROT = 5, WK_MATCH = 6, WK_SKIP = 7 };
+enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL = 4, WK_ROT = 5, WK_MATCH = 6, WK_SKIP = 7, WK_POP = 8, WK_BATCH = 9 };
 
 // ---- small helpers on register arrays -------------------------------------------------
 
@@ -993,6 +993,10 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                      long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream);
+
+// greedy decomposition with one CTA per matrix, for the matrices whose status holds CLASS_U16 (64 < N <= 256)
+cudaError_t run_mw_team(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
+                        int32_t* residual, int32_t* status, long long* work, cudaStream_t stream);
 
 // scoring with one CTA per matrix, for the matrices whose status holds CLASS_U16 (64 < N <= 256)
 cudaError_t run_eval_team(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,

@@ -363,6 +363,12 @@ static cudaError_t launch_mw_mode(Geometry ge, int B, int N, const int32_t* dema
 #undef MOESCHED_GO
 }
 
+// Batches with fewer matrices per SM than this go to the CTA-per-matrix kernel (N > 64). Measured on a
+// B200: N = 256, B = 256 (1.7 per SM): 294 ms against 613 ms for one warp per matrix; N = 128, B = 1024
+// (6.9 per SM): 91 ms against 63 ms -- with that many matrices per SM the warps of different matrices
+// already fill the issue slots and the CTA's barriers only cost.
+constexpr int MW_TEAM_MAX_PER_SM = 4;
+
 cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,
                    int32_t* residual, int32_t* status, long long* work, cudaStream_t stream) {
   const Geometry ge = plan_geometry(N);
@@ -372,11 +378,16 @@ cudaError_t run_mw(int B, int N, const int32_t* demand, int k_max, uint8_t* perm
     // (one CTA each at any N), then the rest as int32 (a 2-CTA cluster above N = 232).
     cudaError_t e = classify_matrices(B, N, demand, status, stream);
     if (e != cudaSuccess) return e;
-    Geometry g16 = ge;
-    g16.cluster = false;
-    g16.wpb = 1;
-    g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
-    e = launch_mw_mode<2>(g16, B, N, demand, k_max, perm, dur, count, residual, status, work, CLASS_U16, stream);
+    if (N > 64 && B < MW_TEAM_MAX_PER_SM * sm_count()) {
+      // few large matrices: one CTA per matrix instead of one warp
+      e = run_mw_team(B, N, demand, k_max, perm, dur, count, residual, status, work, stream);
+    } else {
+      Geometry g16 = ge;
+      g16.cluster = false;
+      g16.wpb = 1;
+      g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
+      e = launch_mw_mode<2>(g16, B, N, demand, k_max, perm, dur, count, residual, status, work, CLASS_U16, stream);
+    }
     if (e != cudaSuccess) return e;
     only_class = CLASS_I32;
   }

@@ -318,4 +318,219 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
   return ok_all;
 }
 
+
+// ---- canonicalisation with one search per WARP, several rows searched at once -----------------------
+//
+// The graph is held as bit matrices in shared memory (cc: rows adjacent to each column, rr: columns
+// adjacent to each row) next to x / mr. A backward search then needs no exchange between warps: the
+// lanes of ONE warp each look after the rows w * 32 + lane, a frontier row contributes the row set of
+// its matched column with two vector loads, and an OR-reduction per word gives the next level. The NW
+// warps of the CTA search the NW lowest rows that could move at the same time, each as if it were the
+// only one. That is exact as long as no searched row moves: a search for row i looks at the rows above
+// i and the current matching only. The results are then taken in row order up to the first row that
+// does move; that warp rotates the matching along its cycle, the searches of the rows behind it are
+// thrown away and the rows that could move are determined anew.
+template <int NW>
+struct TeamSearchShared {
+  static constexpr int NT = 32 * NW;
+  unsigned cc[NT * NW];     // word w of the rows adjacent to column c at cc[c * NW + w]
+  unsigned rr[NT * NW];     // word w of the columns adjacent to row r at rr[r * NW + w]
+  int lvl[NW][NT];          // per warp: stamp of the level at which its search reached a row
+  int res[NW][4];           // per warp: row searched, column found, levels, rows reached
+};
+
+// The k-th lowest member (k = 0 for the lowest) of a set, or -1 if it has no more than k members.
+template <int W>
+__device__ __forceinline__ int kth_member(const unsigned (&m)[W], int k) {
+  int r = -1, seen = 0;
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    const int pc = __popc(m[w]);
+    if (r < 0 && k < seen + pc) {
+      unsigned v = m[w];
+      for (int q = seen; q < k; ++q) v &= v - 1u;
+      r = w * 32 + __ffs(v) - 1;
+    }
+    seen += pc;
+  }
+  return r;
+}
+
+template <int W>
+__device__ __forceinline__ void load_words(const unsigned* p, unsigned (&out)[W]) {
+  if constexpr (W % 4 == 0) {
+#pragma unroll
+    for (int q = 0; q < W / 4; ++q) {
+      const uint4 v = reinterpret_cast<const uint4*>(p)[q];
+      out[4 * q] = v.x; out[4 * q + 1] = v.y; out[4 * q + 2] = v.z; out[4 * q + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int w = 0; w < W; ++w) out[w] = p[w];
+  }
+}
+
+// Backward search from row i among the rows above it (one warp; every lane returns the same values):
+// the lowest column that row i can take in a perfect matching that keeps the rows below i where they
+// are, or -1 if an iteration limit was hit. lvl[r] = stamp + level for every row reached (row i: stamp).
+template <int NW>
+__device__ __forceinline__ int warp_back_search(const TeamShared<NW>& sh, const TeamSearchShared<NW>& ts, int* lvl,
+                                                int stamp, int N, int i, int lane, int& levels, int& reached) {
+  constexpr int W = NW;
+  unsigned anc[W], F[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) anc[w] = F[w] = onehot_word(i, w);
+  if (lane == 0) lvl[i] = stamp;
+  int level = 0;
+  levels = 0;
+  reached = 1;
+  for (int it = 0; it < N; ++it) {
+    unsigned acc[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      if ((F[w] >> lane) & 1u) {
+        const int c = sh.x[w * 32 + lane];
+        unsigned col[W];
+        load_words<W>(ts.cc + c * W, col);
+#pragma unroll
+        for (int q = 0; q < W; ++q) acc[q] |= col[q];
+      }
+    }
+    bool grew = false;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const unsigned a = __reduce_or_sync(FULL, acc[w]) & ge_word(i + 1, w) & ~anc[w];
+      anc[w] |= a;
+      F[w] = a;
+      grew |= a != 0u;
+      reached += __popc(a);
+    }
+    ++levels;
+    if (!grew) break;
+    ++level;
+#pragma unroll
+    for (int w = 0; w < W; ++w)
+      if ((F[w] >> lane) & 1u) lvl[w * 32 + lane] = stamp + level;
+  }
+  __syncwarp();
+  // lowest column adjacent to row i whose row was reached (its own column always qualifies)
+  int jstar = -1;
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    const int c = w * 32 + lane;
+    bool ok = false;
+    if (c < N && ((ts.rr[i * W + w] >> lane) & 1u)) {
+      const int r = sh.mr[c];
+      ok = r >= 0 && test_bit<W>(anc, r);
+    }
+    const unsigned ball = __ballot_sync(FULL, ok);
+    if (jstar < 0 && ball != 0u) jstar = w * 32 + __ffs(ball) - 1;
+  }
+  return jstar;
+}
+
+// Rotation along the alternating cycle found by warp_back_search (same warp, same lvl, same stamp):
+// the row that gives up column jstar takes the column of its successor towards row i, and so on
+// down the levels; row i takes jstar. Returns the highest row moved, or -1 on an inconsistency.
+template <int NW>
+__device__ __forceinline__ int warp_rotate(TeamShared<NW>& sh, const TeamSearchShared<NW>& ts, const int* lvl, int stamp,
+                                           int N, int i, int jstar, int lane, int& steps) {
+  constexpr int W = NW;
+  int cur = sh.mr[jstar];
+  int L = lvl[cur] - stamp;
+  int top = i;
+  if (L <= 0 || L > N) return -1;
+  for (int it = 0; it < N && L > 0; ++it) {
+    int cp = -1;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const int c = w * 32 + lane;
+      bool ok = false;
+      if (c < N && ((ts.rr[cur * W + w] >> lane) & 1u)) {
+        const int r = sh.mr[c];
+        ok = r >= 0 && lvl[r] == stamp + L - 1;
+      }
+      const unsigned ball = __ballot_sync(FULL, ok);
+      if (cp < 0 && ball != 0u) cp = w * 32 + __ffs(ball) - 1;
+    }
+    if (cp < 0) return -1;
+    const int nxt = sh.mr[cp];
+    __syncwarp();
+    if (lane == 0) { sh.mr[cp] = (short)cur; sh.x[cur] = (short)cp; }
+    __syncwarp();
+    top = max(top, cur);
+    cur = nxt;
+    --L;
+    ++steps;
+  }
+  if (cur != i) return -1;
+  if (lane == 0) { sh.mr[jstar] = (short)i; sh.x[i] = (short)jstar; }
+  __syncwarp();
+  return top;
+}
+
+// Lexicographically smallest perfect matching of the graph (ts.cc / ts.rr, m.Rr) over the rows
+// [start, N), given a perfect matching that already equals the answer below `start`; see
+// canonicalise() in common.cuh for the argument. Same result as team_canonicalise. Uniform.
+template <int NW>
+__device__ __forceinline__ bool team_canonicalise_par(TeamShared<NW>& sh, TeamSearchShared<NW>& ts, TeamRed& red, int N,
+                                                      int t, int lane, int warp, bool in, TeamMatch<NW>& m, int& stamp,
+                                                      int start, unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = NW;
+  bool ok_all = true;
+  bool cand = team_is_candidate<NW>(sh, t, lane, warp, in, m);
+  int from = start;
+  for (int guard = 0; guard < N; ++guard) {
+    unsigned todo[W];
+    red.open();
+    red.add_member<W>(cand && t >= from, t, lane);
+    red.close();
+    red.read_set<W>(todo);
+    red.next();
+    if (!any_bit<W>(todo)) break;
+    // a fresh range of level stamps for this round (each warp marks in its own array)
+    if (stamp > 0x7f000000) {
+      __syncthreads();
+#pragma unroll
+      for (int w = 0; w < W; ++w) ts.lvl[w][t] = -1;
+      stamp = 0;
+      __syncthreads();
+    }
+    stamp += N + 2;
+    const int i = kth_member<W>(todo, warp);
+    int jstar = -1, levels = 0, reached = 0;
+    if (i >= 0) jstar = warp_back_search<NW>(sh, ts, ts.lvl[warp], stamp, N, i, lane, levels, reached);
+    if (lane == 0) { ts.res[warp][0] = i; ts.res[warp][1] = jstar; ts.res[warp][2] = levels; ts.res[warp][3] = reached; }
+    __syncthreads();
+    // results in row order, up to the first row that moves
+    int wrot = -1, last_done = from - 1;
+    bool bad = false;
+    for (int w = 0; w < NW; ++w) {
+      const int iw = ts.res[w][0], jw = ts.res[w][1];
+      if (iw < 0) break;
+      if (jw < 0) { bad = true; break; }
+      last_done = iw;
+      if (t == 0) { work[WK_SWEEP]++; work[WK_LEVEL] += ts.res[w][2]; work[WK_POP] += ts.res[w][3]; }
+      if (jw != sh.x[iw]) { wrot = w; break; }
+    }
+    if (bad) { ok_all = false; break; }
+    from = last_done + 1;
+    if (wrot < 0) continue;   // none of the searched rows moves: the matching and the candidates stand
+    if (warp == wrot) {
+      int steps = 0;
+      const int top = warp_rotate<NW>(sh, ts, ts.lvl[warp], stamp, N, ts.res[wrot][0], ts.res[wrot][1], lane, steps);
+      if (lane == 0) { sh.misc[4] = top; sh.misc[5] = steps; }
+    }
+    __syncthreads();
+    if (sh.misc[4] < 0) { ok_all = false; break; }
+    if (t == 0) work[WK_ROT] += sh.misc[5];
+    m.my_x = sh.x[t];
+    m.my_mr = sh.mr[t];
+    cand = team_is_candidate<NW>(sh, t, lane, warp, in, m);
+  }
+  return ok_all;
+}
+
 }  // namespace moesched

@@ -36,8 +36,8 @@ PLAN = {
     ("bvn", 3): 512,
     ("bvn", 4): 64,
     ("bvn", 5): 8,
-    ("mw", 4): 256,
-    ("mw", 5): 32,
+    ("mw", 4): 1024,
+    ("mw", 5): 256,
 }
 
 

@@ -114,8 +114,8 @@ PLAN = {
     1: dict(mw_rows={8: 64}, bvn_rows=64, bvn_prefix=None),
     2: dict(mw_rows={4: 1024, 16: 1024}, bvn_rows=1024, bvn_prefix=None),
     3: dict(mw_rows={8: 128, 16: 128, 64: 4096}, bvn_rows=64, bvn_prefix=None),
-    4: dict(mw_rows={16: 64, 32: 64, 128: 32}, bvn_rows=16, bvn_prefix=None),
-    5: dict(mw_rows={4: 32, 8: 32, 16: 32, 32: 32, 256: 8}, bvn_rows=16, bvn_prefix=40),
+    4: dict(mw_rows={16: 64, 32: 64, 128: 256}, bvn_rows=16, bvn_prefix=None),
+    5: dict(mw_rows={4: 32, 8: 32, 16: 32, 32: 32, 256: 32}, bvn_rows=16, bvn_prefix=40),
 }
 # Complete schedules of many more matrices (configuration 3: 512, 4: 64 Birkhoff and 256 greedy,
 # 5: 8 Birkhoff and 32 greedy, every matching of each) are compared through the oracle's stored

@@ -90,7 +90,7 @@ def test_bvn_complete_schedules_match_the_oracle_digests(cfg, min_rows):
             same_schedules(part, s)
 
 
-@pytest.mark.parametrize("cfg,min_rows", [(4, 128), (5, 16)])
+@pytest.mark.parametrize("cfg,min_rows", [(4, 1024), (5, 256)])
 def test_greedy_largest_budget_matches_the_oracle_digests(cfg, min_rows):
     D = make_demand(cfg)
     d = torch.from_numpy(D).cuda()
