@@ -116,6 +116,41 @@ def schedule_prefix_eval(demand, perm, dur, count, model, threads=1):
     return dict(prefix_overlap_ns=po, prefix_unserved_tokens=pu, status=status)
 
 
+def schedule_order(demand, perm, dur, count, model, threads=1):
+    """Best-of-several order of the matchings on fixed job times (see order_one in the C++ source)."""
+    d = np.ascontiguousarray(demand, dtype=np.int32)
+    B, N, _ = d.shape
+    perm = np.ascontiguousarray(perm, dtype=np.uint8)
+    dur = np.ascontiguousarray(dur, dtype=np.int32)
+    count = np.ascontiguousarray(count, dtype=np.int32)
+    K = perm.shape[1]
+    m = np.array([int(model.get(f, 0)) for f in MODEL_FIELDS], np.int64)
+    order = np.zeros((B, K), np.int32)
+    best = np.zeros(B, np.int64)
+    emission = np.zeros(B, np.int64)
+    rule = np.zeros(B, np.int32)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_schedule_order(B, N, _p(d), K, _p(perm), _p(dur), _p(count), _p(m), _p(order), _p(best),
+                                     _p(emission), _p(rule), _p(status), threads)
+    if rc != 0:
+        raise ValueError("oracle_schedule_order rejected its arguments")
+    return dict(order=order, makespan_ns=best, emission_ns=emission, rule=rule, status=status)
+
+
+def best_budget(count, prefix_overlap_ns, prefix_unserved_tokens, ns_per_unserved_token):
+    count = np.ascontiguousarray(count, dtype=np.int32)
+    po = np.ascontiguousarray(prefix_overlap_ns, dtype=np.int64)
+    pu = np.ascontiguousarray(prefix_unserved_tokens, dtype=np.int64)
+    B, K = po.shape
+    best_k = np.zeros(B, np.int32)
+    best_cost = np.zeros(B, np.int64)
+    rc = lib().oracle_best_budget(B, K, _p(count), _p(po), _p(pu), ctypes.c_int64(int(ns_per_unserved_token)),
+                                  _p(best_k), _p(best_cost))
+    if rc != 0:
+        raise ValueError("oracle_best_budget rejected its arguments")
+    return dict(best_k=best_k, best_cost=best_cost)
+
+
 def ideal_a2a(demand, model):
     d = np.ascontiguousarray(demand, dtype=np.int32)
     B, N, _ = d.shape

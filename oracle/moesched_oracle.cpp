@@ -460,6 +460,112 @@ bool model_ok(const Model& m) {
          m.expert_ps_per_token >= 0 && m.expert_knee_tokens >= 0;
 }
 
+// ---------------------------------------------------------------------------
+// Order of the matchings [Sec. 3.3, last paragraph: with dispatch, compute and combine as the three
+// machines of a flow shop, the order in which the matchings run changes the makespan; the paper
+// leaves the rule open]. Stated here as a best-of-several rule on FIXED job times:
+//   a_k = reconfig + t_k   (dispatch of matching k; the combine stage takes the same time, c_k = a_k)
+//   b_k = comp_k           (its expert batch), both as the replay in emission order gives them.
+// Candidate orders (ties always broken by the lower original index):
+//   0  emission order;
+//   1  Johnson's rule on the first two stages: jobs with a_k <= b_k first, by increasing a_k, then
+//      the others by decreasing b_k;
+//   2  Johnson's rule on the last two stages: jobs with b_k <= a_k first, by increasing b_k, then the
+//      others by decreasing a_k;
+//   3  light ends: by increasing a_k, placed alternately at the front and at the back, so that the
+//      shortest transfers open and close the schedule (a compute-bound schedule lasts
+//      a_first + sum b + a_last);
+//   4  longest expert batch first: by decreasing b_k.
+// Each candidate is run through the three-stage recurrence of eval_one on these times; the one with
+// the smallest makespan wins, the lower rule number on ties. Rule 0 is among them, so the result is
+// never worse than the emission order. The times are exact for the reordered schedule whenever no
+// pair with demand occurs in two matchings (a greedy schedule repeats a pair only as an idle,
+// zero-weight filler; moving such a filler ahead of the matching that serves the pair would let it
+// carry tokens in a replay, so the reordered schedule is scored again by oracle_schedule_eval where
+// the exact figure is wanted).
+// Outputs per matrix: order[pos] = original index of the matching that runs at position pos
+// (entries >= count are -1), the makespan of that order and of the emission order on the fixed
+// times, the winning rule. A schedule that oracle_schedule_eval rejects gives status BAD_INPUT,
+// order -1 everywhere, both makespans 0 and rule 0.
+// ---------------------------------------------------------------------------
+i64 fixed_times_makespan(const std::vector<int>& ord, const std::vector<i64>& a, const std::vector<i64>& b) {
+  i64 dsp = 0, cmp = 0, cmb = 0;
+  for (int k : ord) {
+    dsp = dsp + a[k];
+    cmp = std::max(dsp, cmp) + b[k];
+    cmb = std::max(cmp, cmb) + a[k];
+  }
+  return cmb;
+}
+
+void order_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t* dur, const Model& m,
+               int k_stride, int32_t* order, i64* best_ns, i64* emission_ns, int32_t* rule, int32_t* status) {
+  for (int k = 0; k < k_stride; ++k) order[k] = -1;
+  *best_ns = *emission_ns = 0;
+  *rule = 0;
+  i64 o, s, in, it, un;
+  eval_one(N, D, K, perm, dur, m, &o, &s, &in, &it, &un, status);
+  if (*status != ST_OK) return;
+  // job times from the replay in emission order
+  std::vector<i64> a(K), b(K);
+  std::vector<i64> R(D, D + (size_t)N * N);
+  for (int k = 0; k < K; ++k) {
+    i64 g = 0;
+    for (int i = 0; i < N; ++i) {
+      i64& x = R[i * N + perm[(size_t)k * N + i]];
+      i64 served = std::min<i64>(dur[k], x);
+      x -= served;
+      g = std::max(g, served);
+    }
+    a[k] = m.reconfig_ns + cdiv((i64)dur[k] * m.bytes_per_token * 8, m.link_gbps);
+    b[k] = batch_time(m, g);
+  }
+  std::vector<std::vector<int>> cand(5);
+  std::vector<int> idx(K);
+  std::iota(idx.begin(), idx.end(), 0);
+  cand[0] = idx;
+  {
+    std::vector<int> head, tail;
+    for (int k : idx) (a[k] <= b[k] ? head : tail).push_back(k);
+    std::stable_sort(head.begin(), head.end(), [&](int p, int q) { return a[p] < a[q]; });
+    std::stable_sort(tail.begin(), tail.end(), [&](int p, int q) { return b[p] > b[q]; });
+    cand[1] = head;
+    cand[1].insert(cand[1].end(), tail.begin(), tail.end());
+  }
+  {
+    std::vector<int> head, tail;
+    for (int k : idx) (b[k] <= a[k] ? head : tail).push_back(k);
+    std::stable_sort(head.begin(), head.end(), [&](int p, int q) { return b[p] < b[q]; });
+    std::stable_sort(tail.begin(), tail.end(), [&](int p, int q) { return a[p] > a[q]; });
+    cand[2] = head;
+    cand[2].insert(cand[2].end(), tail.begin(), tail.end());
+  }
+  {
+    std::vector<int> by_a(idx);
+    std::stable_sort(by_a.begin(), by_a.end(), [&](int p, int q) { return a[p] < a[q]; });
+    cand[3].assign(K, 0);
+    int front = 0, back = K - 1;
+    for (int r = 0; r < K; ++r) {
+      if (r % 2 == 0) cand[3][front++] = by_a[r];
+      else cand[3][back--] = by_a[r];
+    }
+  }
+  {
+    cand[4] = idx;
+    std::stable_sort(cand[4].begin(), cand[4].end(), [&](int p, int q) { return b[p] > b[q]; });
+  }
+  int win = 0;
+  i64 best = 0;
+  for (int c = 0; c < 5; ++c) {
+    const i64 mk = fixed_times_makespan(cand[c], a, b);
+    if (c == 0) { *emission_ns = mk; best = mk; }
+    else if (mk < best) { best = mk; win = c; }
+  }
+  for (int k = 0; k < K; ++k) order[k] = cand[win][k];
+  *best_ns = best;
+  *rule = win;
+}
+
 template <class F>
 void parallel_for(int B, int threads, F f) {
   if (threads <= 1 || B <= 1) { for (int b = 0; b < B; ++b) f(b); return; }
@@ -558,6 +664,61 @@ int oracle_schedule_prefix_eval(int B, int N, const int32_t* demand, int k_strid
     }
     status[b] = ST_OK;
   });
+  return 0;
+}
+
+// See order_one above. order: [B][k_stride] int32; best_ns, emission_ns: [B] int64; rule, status: [B] int32.
+int oracle_schedule_order(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm,
+                          const int32_t* dur, const int32_t* count, const int64_t* model, int32_t* order,
+                          int64_t* best_ns, int64_t* emission_ns, int32_t* rule, int32_t* status, int threads) {
+  if (B < 0 || N < 1 || N > 256 || k_stride < 1 || !demand || !perm || !dur || !count || !model || !order ||
+      !best_ns || !emission_ns || !rule || !status)
+    return -1;
+  Model m = {model[0], model[1], model[2], model[3], model[4], model[5]};
+  if (!model_ok(m)) return -1;
+  const size_t NN = (size_t)N * N;
+  parallel_for(B, threads, [&](int b) {
+    int32_t* ob = order + (size_t)b * k_stride;
+    const int K = count[b];
+    if (K < 0 || K > k_stride) {
+      for (int k = 0; k < k_stride; ++k) ob[k] = -1;
+      best_ns[b] = emission_ns[b] = 0;
+      rule[b] = 0;
+      status[b] = ST_BAD_INPUT;
+      return;
+    }
+    i64 best, emi;
+    order_one(N, demand + b * NN, K, perm + (size_t)b * k_stride * N, dur + (size_t)b * k_stride, m, k_stride, ob,
+              &best, &emi, rule + b, status + b);
+    best_ns[b] = best;
+    emission_ns[b] = emi;
+  });
+  return 0;
+}
+
+// Budget choice [Sec. 3.2 / 3.3: how many matchings to run]: with the prefix scores of a schedule
+// (oracle_schedule_prefix_eval) and a price in ns per token left unserved, the number of matchings
+// k in 1..count that minimises  prefix_overlap_ns[k-1] + ns_per_unserved_token * prefix_unserved[k-1]
+// (price 0 .. 2^15 ns per token, so that the sum stays within 63 bits);
+// the smallest such k on ties. count = 0, or a schedule whose prefix entries are -1 (rejected), gives
+// best_k = 0 and best_cost = 0.
+int oracle_best_budget(int B, int k_stride, const int32_t* count, const int64_t* prefix_overlap_ns,
+                       const int64_t* prefix_unserved_tokens, int64_t ns_per_unserved_token, int32_t* best_k,
+                       int64_t* best_cost) {
+  if (B < 0 || k_stride < 1 || !count || !prefix_overlap_ns || !prefix_unserved_tokens || !best_k || !best_cost ||
+      ns_per_unserved_token < 0 || ns_per_unserved_token > (1LL << 15))
+    return -1;
+  for (int b = 0; b < B; ++b) {
+    best_k[b] = 0;
+    best_cost[b] = 0;
+    const int K = std::min(std::max(count[b], 0), k_stride);
+    for (int k = 0; k < K; ++k) {
+      const i64 o = prefix_overlap_ns[(size_t)b * k_stride + k], u = prefix_unserved_tokens[(size_t)b * k_stride + k];
+      if (o < 0 || u < 0) { best_k[b] = 0; best_cost[b] = 0; break; }
+      const i64 cost = o + ns_per_unserved_token * u;
+      if (k == 0 || cost < best_cost[b]) { best_cost[b] = cost; best_k[b] = k + 1; }
+    }
+  }
   return 0;
 }
 
