@@ -228,6 +228,57 @@ int moesched_schedule_prefix_eval(int B, int N, const int32_t* d_demand, int k_s
                                   int64_t* d_prefix_unserved_tokens, void* stream);
 
 /*
+ * Order of the matchings (paper Sec. 3.3, last paragraph: dispatch, expert compute and combine are
+ * the three machines of a flow shop and the order of the matchings changes the makespan; the paper
+ * leaves the rule open). This entry point chooses the best of five orders on FIXED job times
+ *   a_k = reconfig_ns + t_k (dispatch; the combine stage takes the same time),  b_k = comp_k,
+ * both as the replay in emission order gives them (see moesched_schedule_eval). Candidates, ties
+ * always by the lower original index: 0 the emission order; 1 Johnson's rule on stages one and two
+ * (jobs with a <= b first by increasing a, then the rest by decreasing b); 2 Johnson's rule on stages
+ * two and three (b <= a first by increasing b, then the rest by decreasing a); 3 increasing a, placed
+ * alternately at the front and at the back (the shortest transfers open and close the schedule);
+ * 4 decreasing b. Each is run through the three-stage recurrence; the shortest wins, the lower rule
+ * number on ties, so the result is never worse than the emission order. The fixed times are exact
+ * for the reordered schedule when no pair with demand occurs in two matchings; a greedy schedule
+ * repeats a pair only as an idle filler, and scoring the reordered schedule (moesched_schedule_permute,
+ * then moesched_schedule_eval) gives the exact figure where it matters.
+ *
+ *   k_stride          in   1 .. MOESCHED_ORDER_MAX_K
+ *   d_demand ... h_model   as in moesched_schedule_eval
+ *   d_order           out  [B][k_stride] int32: d_order[b][p] = original index of the matching that
+ *                          runs at position p; -1 for p >= count[b] and for rejected schedules
+ *   d_makespan_ns     out  [B] int64 makespan of the chosen order on the fixed job times
+ *   d_emission_ns     out  [B] int64 the same for the emission order (= makespan_overlap_ns)
+ *   d_rule            out  [B] int32 number of the winning candidate
+ *   d_status          out  [B] int32 OK, or BAD_INPUT (a schedule moesched_schedule_eval rejects)
+ *   d_scratch         tmp  moesched_order_scratch_bytes(B, k_stride) bytes, 8-byte aligned
+ */
+#define MOESCHED_ORDER_MAX_K 1024
+size_t moesched_order_scratch_bytes(int B, int k_stride);
+int moesched_schedule_order(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                            const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                            int32_t* d_order, int64_t* d_makespan_ns, int64_t* d_emission_ns, int32_t* d_rule,
+                            int32_t* d_status, void* d_scratch, void* stream);
+
+/* The schedule in a new order: d_perm_out[b][p] = d_perm[b][d_order[b][p]] and the same for the
+ * durations, for every position whose order entry lies in 0 .. k_stride-1; other positions are left
+ * untouched. The output arrays must not overlap the input arrays. */
+int moesched_schedule_permute(int B, int N, int k_stride, const uint8_t* d_perm, const int32_t* d_dur,
+                              const int32_t* d_order, uint8_t* d_perm_out, int32_t* d_dur_out, void* stream);
+
+/*
+ * Budget choice (paper Sec. 3.2 / 3.3: how many matchings are worth running): from the prefix scores of
+ * moesched_schedule_prefix_eval and a price in ns per token left unserved (0 .. 2^15), the number of
+ * matchings k in 1 .. count[b] that minimises
+ *   d_prefix_overlap_ns[b][k-1] + ns_per_unserved_token * d_prefix_unserved_tokens[b][k-1],
+ * the smallest such k on ties. d_best_k [B] int32, d_best_cost [B] int64; both 0 for an empty
+ * schedule or one whose prefix entries are -1 (rejected).
+ */
+int moesched_best_budget(int B, int k_stride, const int32_t* d_count, const int64_t* d_prefix_overlap_ns,
+                         const int64_t* d_prefix_unserved_tokens, int64_t ns_per_unserved_token,
+                         int32_t* d_best_k, int64_t* d_best_cost, void* stream);
+
+/*
  * Idealised congestion-free all-to-all (paper Sec. 4.1 "Comparisons": the best completion time
  * any fabric could reach for the matrix), the yardstick the decomposed schedules are compared
  * with. Every port sends and receives at line rate, so one exchange

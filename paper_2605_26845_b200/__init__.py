@@ -50,9 +50,11 @@ def load_library():
         lib.moesched_workspace_bytes.restype = ctypes.c_size_t
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
                      "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
-                     "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error"):
+                     "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error",
+                     "moesched_schedule_order", "moesched_schedule_permute", "moesched_best_budget"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
+        lib.moesched_order_scratch_bytes.restype = ctypes.c_size_t
         lib.moesched_probe_int_ops.restype = ctypes.c_longlong
         _lib = lib
     return _lib
@@ -311,6 +313,67 @@ def schedule_eval(demand, perm, dur, count, model=None, out=None, status=None, p
         res["prefix_overlap_ns"], res["prefix_unserved_tokens"] = pre[0], pre[1]
     res["status"] = status
     return res
+
+
+ORDER_MAX_K = 1024
+
+
+def schedule_order(demand, perm, dur, count, model=None) -> dict:
+    """Best of five orders of the matchings on the job times of the emission-order replay (paper
+    Sec. 3.3). Returns 'order' [B, k_stride] int32 (position -> original index, -1 beyond count),
+    'makespan_ns', 'emission_ns' [B] int64, 'rule', 'status' [B] int32."""
+    lib = load_library()
+    demand = _check_demand(demand)
+    perm = _dev(perm, torch.uint8, "perm")
+    dur = _dev(dur, torch.int32, "dur")
+    count = _dev(count, torch.int32, "count")
+    B, N, _ = demand.shape
+    K = int(perm.shape[1])
+    if perm.dim() != 3 or perm.shape[0] != B or perm.shape[2] != N or dur.shape != perm.shape[:2]:
+        raise MoeschedError("perm must be [B, k_stride, N] and dur [B, k_stride]")
+    dev = demand.device
+    m = _model(model)
+    order = torch.empty((B, K), dtype=torch.int32, device=dev)
+    times = torch.empty((2, B), dtype=torch.int64, device=dev)
+    small = torch.empty((2, B), dtype=torch.int32, device=dev)
+    scratch = torch.empty(max(8, int(lib.moesched_order_scratch_bytes(B, K))), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib.moesched_schedule_order(B, N, _ptr(demand), K, _ptr(perm), _ptr(dur), _ptr(count), ctypes.byref(m),
+                                         _ptr(order), _ptr(times[0]), _ptr(times[1]), _ptr(small[0]), _ptr(small[1]),
+                                         _ptr(scratch), _stream(dev))
+    _check(rc, "moesched_schedule_order")
+    return {"order": order, "makespan_ns": times[0], "emission_ns": times[1], "rule": small[0], "status": small[1]}
+
+
+def schedule_permute(perm, dur, order):
+    """(perm, dur) with the matchings in the given order; positions whose order entry is -1 hold zeros."""
+    lib = load_library()
+    perm = _dev(perm, torch.uint8, "perm")
+    dur = _dev(dur, torch.int32, "dur")
+    order = _dev(order, torch.int32, "order")
+    B, K, N = perm.shape
+    perm_out, dur_out = torch.zeros_like(perm), torch.zeros_like(dur)
+    with torch.cuda.device(perm.device):
+        rc = lib.moesched_schedule_permute(B, N, K, _ptr(perm), _ptr(dur), _ptr(order), _ptr(perm_out), _ptr(dur_out),
+                                           _stream(perm.device))
+    _check(rc, "moesched_schedule_permute")
+    return perm_out, dur_out
+
+
+def best_budget(count, prefix_overlap_ns, prefix_unserved_tokens, ns_per_unserved_token) -> dict:
+    """Number of matchings (1..count) minimising prefix makespan + price * unserved tokens."""
+    lib = load_library()
+    count = _dev(count, torch.int32, "count")
+    po = _dev(prefix_overlap_ns, torch.int64, "prefix_overlap_ns")
+    pu = _dev(prefix_unserved_tokens, torch.int64, "prefix_unserved_tokens")
+    B, K = po.shape
+    best_k = torch.empty(B, dtype=torch.int32, device=po.device)
+    best_cost = torch.empty(B, dtype=torch.int64, device=po.device)
+    with torch.cuda.device(po.device):
+        rc = lib.moesched_best_budget(B, K, _ptr(count), _ptr(po), _ptr(pu), ctypes.c_int64(int(ns_per_unserved_token)),
+                                      _ptr(best_k), _ptr(best_cost), _stream(po.device))
+    _check(rc, "moesched_best_budget")
+    return {"best_k": best_k, "best_cost": best_cost}
 
 
 class Path:

@@ -150,6 +150,67 @@ int moesched_schedule_prefix_eval(int B, int N, const int32_t* d_demand, int k_s
                             d_status, d_prefix_overlap_ns, d_prefix_unserved_tokens, stream);
 }
 
+size_t moesched_order_scratch_bytes(int B, int k_stride) {
+  if (B < 0 || k_stride < 1 || k_stride > MOESCHED_ORDER_MAX_K) return 0;
+  return (size_t)B * (2 * (size_t)k_stride + 5) * sizeof(int64_t) + (((size_t)B * sizeof(int32_t) + 7) & ~(size_t)7);
+}
+
+int moesched_schedule_order(int B, int N, const int32_t* d_demand, int k_stride, const uint8_t* d_perm,
+                            const int32_t* d_dur, const int32_t* d_count, const moesched_model_t* h_model,
+                            int32_t* d_order, int64_t* d_makespan_ns, int64_t* d_emission_ns, int32_t* d_rule,
+                            int32_t* d_status, void* d_scratch, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_stride < 1 || k_stride > MOESCHED_ORDER_MAX_K) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_demand || !d_perm || !d_dur || !d_count || !h_model || !d_order || !d_makespan_ns || !d_emission_ns ||
+      !d_rule || !d_status || !d_scratch)
+    return MOESCHED_EINVAL;
+  if (!aligned4(d_demand) || !aligned4(d_dur) || !aligned4(d_count) || !aligned4(d_order) || !aligned4(d_rule) ||
+      !aligned4(d_status) || !aligned8(d_makespan_ns) || !aligned8(d_emission_ns) || !aligned8(d_scratch))
+    return MOESCHED_EINVAL;
+  const moesched_model_t m = *h_model;
+  if (!model_in_range(m)) return MOESCHED_EINVAL;
+  // scratch: job times [B][k_stride] x 2, five score arrays [B], the scoring status [B]
+  long long* leg = static_cast<long long*>(d_scratch);
+  long long* comp = leg + (size_t)B * k_stride;
+  long long* scores = comp + (size_t)B * k_stride;
+  int32_t* eval_status = reinterpret_cast<int32_t*>(scores + (size_t)5 * B);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = run_eval(B, N, d_demand, k_stride, d_perm, d_dur, d_count, m, scores, scores + B, scores + 2 * (size_t)B,
+                           scores + 3 * (size_t)B, scores + 4 * (size_t)B, eval_status, leg, comp, st, true);
+  if (e == cudaSuccess)
+    e = run_order(B, k_stride, leg, comp, d_count, eval_status, d_order, reinterpret_cast<long long*>(d_makespan_ns),
+                  reinterpret_cast<long long*>(d_emission_ns), d_rule, d_status, st);
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_schedule_permute(int B, int N, int k_stride, const uint8_t* d_perm, const int32_t* d_dur,
+                              const int32_t* d_order, uint8_t* d_perm_out, int32_t* d_dur_out, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_stride < 1) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_perm || !d_dur || !d_order || !d_perm_out || !d_dur_out) return MOESCHED_EINVAL;
+  if (!aligned4(d_dur) || !aligned4(d_order) || !aligned4(d_dur_out) || d_perm == d_perm_out || d_dur == d_dur_out)
+    return MOESCHED_EINVAL;
+  cudaError_t e = run_permute(B, N, k_stride, d_perm, d_dur, d_order, d_perm_out, d_dur_out,
+                              static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+int moesched_best_budget(int B, int k_stride, const int32_t* d_count, const int64_t* d_prefix_overlap_ns,
+                         const int64_t* d_prefix_unserved_tokens, int64_t ns_per_unserved_token,
+                         int32_t* d_best_k, int64_t* d_best_cost, void* stream) {
+  if (B < 0 || k_stride < 1 || ns_per_unserved_token < 0 || ns_per_unserved_token > (1LL << 15)) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_count || !d_prefix_overlap_ns || !d_prefix_unserved_tokens || !d_best_k || !d_best_cost) return MOESCHED_EINVAL;
+  if (!aligned4(d_count) || !aligned4(d_best_k) || !aligned8(d_prefix_overlap_ns) ||
+      !aligned8(d_prefix_unserved_tokens) || !aligned8(d_best_cost))
+    return MOESCHED_EINVAL;
+  cudaError_t e = run_best_budget(B, k_stride, d_count, reinterpret_cast<const long long*>(d_prefix_overlap_ns),
+                                  reinterpret_cast<const long long*>(d_prefix_unserved_tokens),
+                                  (long long)ns_per_unserved_token, d_best_k,
+                                  reinterpret_cast<long long*>(d_best_cost), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
 int moesched_ideal_a2a(int B, int N, const int32_t* d_demand, const moesched_model_t* h_model, int64_t* d_comm_ns,
                        int64_t* d_makespan_ns, int32_t* d_status, void* stream) {
   if (B < 0 || N < 1 || N > MOESCHED_MAX_N) return MOESCHED_EINVAL;

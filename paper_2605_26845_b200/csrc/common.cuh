@@ -992,7 +992,16 @@ inline int bvn_scratch_stride(int N) { return (N + 7) / 8 * 8; }
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
-                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream);
+                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream, bool jobs = false);
+// matching order and budget choice (order_kernel.cu)
+cudaError_t run_order(int B, int k_stride, const long long* leg, const long long* comp, const int32_t* count,
+                      const int32_t* eval_status, int32_t* order, long long* best_ns, long long* emission_ns,
+                      int32_t* rule, int32_t* status, cudaStream_t stream);
+cudaError_t run_permute(int B, int N, int k_stride, const uint8_t* perm, const int32_t* dur, const int32_t* order,
+                        uint8_t* perm_out, int32_t* dur_out, cudaStream_t stream);
+cudaError_t run_best_budget(int B, int k_stride, const int32_t* count, const long long* prefix_overlap,
+                            const long long* prefix_unserved, long long price, int32_t* best_k, long long* best_cost,
+                            cudaStream_t stream);
 
 // greedy decomposition with one CTA per matrix, for the matrices whose status holds CLASS_U16 (64 < N <= 256)
 cudaError_t run_mw_team(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* dur, int32_t* count,

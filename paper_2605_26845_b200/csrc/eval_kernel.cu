@@ -59,9 +59,11 @@ __device__ __forceinline__ Packed<CPL> load_dest(const uint8_t* row, int lane, i
 
 // PREFIX: also write, after every matching k, the overlap makespan and the unserved tokens of the
 // schedule cut after k+1 matchings (entries beyond count, or all entries of a bad schedule, are -1).
+// JOBS (with PREFIX): the two per-matching arrays receive instead the job times of matching k in the
+// three-stage flow shop: reconfiguration + transfer time, and the time of its expert batch.
 // MODE 0: demand in this CTA's shared memory as int32; 1: split over a 2-CTA cluster; 2: held as
 // 16-bit entries (matrices the pre-pass classified as narrow). only_class as in the greedy kernel.
-template <int CPL, int MODE, bool PREFIX>
+template <int CPL, int MODE, bool PREFIX, bool JOBS = false>
 __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_stride,
                                                    const uint8_t* __restrict__ perm, const int32_t* __restrict__ dur,
                                                    const int32_t* __restrict__ count, moesched_model_t model,
@@ -199,8 +201,8 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
           if (lane >= o) run += up;
         }
         if (mine) {
-          prefix_overlap[(size_t)b * k_stride + k0 + lane] = cmb_mine;
-          prefix_unserved[(size_t)b * k_stride + k0 + lane] = total - (served_sum + run);
+          prefix_overlap[(size_t)b * k_stride + k0 + lane] = JOBS ? leg_mine : cmb_mine;
+          prefix_unserved[(size_t)b * k_stride + k0 + lane] = JOBS ? comp_mine : total - (served_sum + run);
         }
         served_sum += __shfl_sync(FULL, run, 31);
       }
@@ -242,11 +244,15 @@ static cudaError_t launch_eval_mode(const Geometry& ge, int B, int N, const int3
                                     const moesched_model_t& model, long long* overlap, long long* serial,
                                     long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
                                     long long* prefix_overlap, long long* prefix_unserved, int only_class,
-                                    cudaStream_t stream) {
+                                    bool jobs, cudaStream_t stream) {
   const bool prefix = prefix_overlap != nullptr;
   const FastDiv by_gbps = make_fastdiv(model.link_gbps);
 #define MOESCHED_GO(C)                                                                                             \
   do {                                                                                                             \
+    if (prefix && jobs)                                                                                            \
+      return launch_warp_kernel(eval_kernel<C, MODE, true, true>, ge, B, stream, B, N, ge.S, demand, k_stride,     \
+                                perm, dur, count, model, by_gbps, overlap, serial, idle_ns, idle_tok, unserved,   \
+                                status, prefix_overlap, prefix_unserved, only_class);                              \
     if (prefix)                                                                                                    \
       return launch_warp_kernel(eval_kernel<C, MODE, true>, ge, B, stream, B, N, ge.S, demand, k_stride, perm,     \
                                 dur, count, model, by_gbps, overlap, serial, idle_ns, idle_tok, unserved,         \
@@ -267,7 +273,7 @@ static cudaError_t launch_eval_mode(const Geometry& ge, int B, int N, const int3
 cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const uint8_t* perm, const int32_t* dur,
                      const int32_t* count, const moesched_model_t& model, long long* overlap, long long* serial,
                      long long* idle_ns, long long* idle_tok, long long* unserved, int32_t* status,
-                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream) {
+                     long long* prefix_overlap, long long* prefix_unserved, cudaStream_t stream, bool jobs) {
   const Geometry ge = plan_geometry(N);
   int only_class = 0;
   if (N >= 48) {
@@ -285,16 +291,16 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
       g16.wpb = 1;
       g16.smem = warp_smem_bytes16(N, g16.S, g16.cpl);
       e = launch_eval_mode<2>(g16, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns,
-                              idle_tok, unserved, status, prefix_overlap, prefix_unserved, CLASS_U16, stream);
+                              idle_tok, unserved, status, prefix_overlap, prefix_unserved, CLASS_U16, jobs, stream);
     }
     if (e != cudaSuccess) return e;
     only_class = CLASS_I32;
   }
   if (ge.cluster)
     return launch_eval_mode<1>(ge, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns,
-                               idle_tok, unserved, status, prefix_overlap, prefix_unserved, only_class, stream);
+                               idle_tok, unserved, status, prefix_overlap, prefix_unserved, only_class, jobs, stream);
   return launch_eval_mode<0>(ge, B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok,
-                             unserved, status, prefix_overlap, prefix_unserved, only_class, stream);
+                             unserved, status, prefix_overlap, prefix_unserved, only_class, jobs, stream);
 }
 
 }  // namespace moesched
