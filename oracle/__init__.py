@@ -178,6 +178,23 @@ def sinkhorn_scale(demand, iters, smooth, scale_bits, threads=1):
     return dict(scaled=scaled, fixed=fixed, stretch=stretch, row_err=row_err, status=status)
 
 
+def bvn_real_decompose(matrix, k_max, tol=1e-12, threads=1):
+    """Real-valued Birkhoff-von Neumann decomposition (see bvn_real_one in the C++ source)."""
+    a = np.ascontiguousarray(matrix, dtype=np.float64)
+    B, N, _ = a.shape
+    perm = np.zeros((B, k_max, N), np.uint8)
+    lam = np.zeros((B, k_max), np.float64)
+    count = np.zeros(B, np.int32)
+    total = np.zeros(B, np.float64)
+    left = np.zeros(B, np.float64)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_bvn_real_decompose(B, N, _p(a), ctypes.c_double(tol), int(k_max), _p(perm), _p(lam), _p(count),
+                                         _p(total), _p(left), _p(status), threads)
+    if rc != 0:
+        raise ValueError("oracle_bvn_real_decompose rejected its arguments")
+    return dict(perm=perm, lam=lam, count=count, sum_lambda=total, max_left=left, status=status)
+
+
 def sinkhorn_durations(coef, count, stretch, scale_bits):
     coef = np.ascontiguousarray(coef, dtype=np.int32)
     count = np.ascontiguousarray(count, dtype=np.int32)

@@ -566,6 +566,57 @@ void order_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_
   *rule = win;
 }
 
+// ---------------------------------------------------------------------------
+// Birkhoff-von Neumann decomposition of a real-valued matrix [Sec. 3.1: A = sum_k lambda_k P_k for a
+// doubly stochastic A; Sec. 4.2 speaks of its coefficients, "around 0.03" on an 8 x 8 matrix]. The
+// input is what Sinkhorn-Knopp scaling returns, doubly stochastic only up to the error of its last
+// sweep, so two things the integer version does not need are stated here: entries at or below `tol`
+// count as zero (on input, and after each subtraction), and the loop also ends when the support has
+// no perfect matching left. Each step: the lexicographically smallest perfect matching of the support,
+// lambda = its smallest entry, subtracted along the matching. All arithmetic is single IEEE double
+// operations in a fixed order. sum_lambda = ((lambda_0 + lambda_1) + ...) in that order; max_left =
+// the largest entry remaining; status OK when nothing remains, TRUNCATED otherwise, BAD_INPUT for a
+// negative or NaN entry.
+// ---------------------------------------------------------------------------
+void bvn_real_one(int N, const double* Min, double tol, int k_max, uint8_t* perm, double* lambda,
+                  int32_t* count, double* sum_lambda, double* max_left, int32_t* status) {
+  const size_t NN = (size_t)N * N;
+  std::vector<double> Wm(NN);
+  *count = 0;
+  *sum_lambda = 0.0;
+  *max_left = 0.0;
+  for (size_t e = 0; e < NN; ++e) {
+    if (!(Min[e] >= 0.0)) { *status = ST_BAD_INPUT; return; }
+    Wm[e] = Min[e] > tol ? Min[e] : 0.0;
+  }
+  std::vector<i64> supp(NN);
+  std::vector<int> pi(N);
+  double total = 0.0;
+  int k = 0;
+  while (k < k_max) {
+    bool any = false;
+    for (size_t e = 0; e < NN; ++e) { supp[e] = Wm[e] > 0.0 ? 1 : 0; any = any || supp[e]; }
+    if (!any) break;
+    if (!t1_support_perm(N, supp.data(), pi.data())) break;   // no perfect matching on what is left
+    double lam = Wm[pi[0]];
+    for (int i = 0; i < N; ++i) lam = std::min(lam, Wm[i * N + pi[i]]);
+    for (int i = 0; i < N; ++i) {
+      double nv = Wm[i * N + pi[i]] - lam;
+      Wm[i * N + pi[i]] = nv > tol ? nv : 0.0;
+    }
+    for (int i = 0; i < N; ++i) perm[(size_t)k * N + i] = (uint8_t)pi[i];
+    lambda[k] = lam;
+    total = total + lam;
+    ++k;
+  }
+  double left = 0.0;
+  for (size_t e = 0; e < NN; ++e) left = std::max(left, Wm[e]);
+  *count = k;
+  *sum_lambda = total;
+  *max_left = left;
+  *status = left > 0.0 ? ST_TRUNCATED : ST_OK;
+}
+
 template <class F>
 void parallel_for(int B, int threads, F f) {
   if (threads <= 1 || B <= 1) { for (int b = 0; b < B; ++b) f(b); return; }
@@ -828,6 +879,21 @@ int oracle_sinkhorn_scale(int B, int N, const int32_t* demand, int iters, double
     stretch[b] = st;
     row_err[b] = err;
     status[b] = dropped ? ST_TRUNCATED : ST_OK;
+  });
+  return 0;
+}
+
+// See bvn_real_one above. matrix [B][N][N] double, perm [B][k_max][N], lambda [B][k_max] double.
+int oracle_bvn_real_decompose(int B, int N, const double* matrix, double tol, int k_max, uint8_t* perm,
+                              double* lambda, int32_t* count, double* sum_lambda, double* max_left,
+                              int32_t* status, int threads) {
+  if (B < 0 || N < 1 || N > 256 || k_max < 1 || !(tol >= 0.0) || !matrix || !perm || !lambda || !count ||
+      !sum_lambda || !max_left || !status)
+    return -1;
+  const size_t NN = (size_t)N * N;
+  parallel_for(B, threads, [&](int b) {
+    bvn_real_one(N, matrix + b * NN, tol, k_max, perm + (size_t)b * k_max * N, lambda + (size_t)b * k_max, count + b,
+                 sum_lambda + b, max_left + b, status + b);
   });
   return 0;
 }

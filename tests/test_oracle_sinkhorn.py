@@ -140,3 +140,71 @@ def test_sinkhorn_then_birkhoff_serves_all_demand_with_many_small_matchings():
     port = np.maximum(D.sum(1).max(1), D.sum(2).max(1))
     total = np.array([dur[b, :v["count"][b]].sum() for b in range(D.shape[0])])
     assert (total >= port).all()
+
+
+# ---- real-valued Birkhoff-von Neumann decomposition (paper Sec. 3.1: A = sum_k lambda_k P_k) ----
+
+def test_real_bvn_on_dyadic_matrices_is_the_integer_decomposition_scaled():
+    """For entries that are integers over a power of two every subtraction is exact, so the real-valued
+    decomposition must reproduce the (separately pinned) integer one: same matchings, lambda = c / 2^s."""
+    for N, seed in ((5, 1), (8, 2), (16, 3), (33, 4)):
+        D = random_matrices(4, N, seed=seed, kind="uniform", high=40, zero_frac=0.4)
+        v = oracle.bvn_decompose(D, bvn_capacity(N))
+        assert (v["status"] == 0).all()
+        T = v["aug"].sum(2)[:, 0]
+        scale = 2.0 ** 12
+        r = oracle.bvn_real_decompose(v["aug"] / scale, bvn_capacity(N), tol=0.0)
+        assert (r["status"] == 0).all() and (r["count"] == v["count"]).all() and (r["max_left"] == 0).all()
+        for b in range(4):
+            K = v["count"][b]
+            assert (r["perm"][b, :K] == v["perm"][b, :K]).all()
+            assert (r["lam"][b, :K] == v["coef"][b, :K] / scale).all()
+            assert r["sum_lambda"][b] == T[b] / scale                 # sum of the coefficients = the common line sum
+
+
+def test_real_bvn_closed_forms_and_reconstruction():
+    N = 8
+    J = np.full((1, N, N), 1.0 / N)
+    r = oracle.bvn_real_decompose(J, 100, tol=0.0)
+    assert r["count"][0] == N and (r["lam"][0, :N] == 1.0 / N).all() and r["sum_lambda"][0] == 1.0
+    assert (r["perm"][0, 0] == np.arange(N)).all() and r["status"][0] == 0
+    P = np.zeros((1, N, N))
+    P[0, np.arange(N), np.roll(np.arange(N), 3)] = 1.0
+    r = oracle.bvn_real_decompose(P, 100)
+    assert r["count"][0] == 1 and r["lam"][0, 0] == 1.0 and (r["perm"][0, 0] == np.roll(np.arange(N), 3)).all()
+    # a scaled demand matrix: the pieces add up to the input, up to what is reported as left over
+    D = make_demand(1, 6)
+    sk = oracle.sinkhorn_scale(D, 200, 0.5, 20)
+    tol = 1e-9
+    r = oracle.bvn_real_decompose(sk["scaled"], bvn_capacity(N), tol=tol)
+    for b in range(6):
+        K = r["count"][b]
+        rebuilt = np.zeros((N, N))
+        for k in range(K):
+            rebuilt[np.arange(N), r["perm"][b, k]] += r["lam"][b, k]
+            assert sorted(r["perm"][b, k]) == list(range(N)) and r["lam"][b, k] > tol
+        gap = sk["scaled"][b] - rebuilt
+        assert gap.min() > -1e-12 and gap.max() <= max(r["max_left"][b], tol) + 1e-12
+        assert K <= bvn_capacity(N)
+        assert abs(r["sum_lambda"][b] - r["lam"][b, :K].sum()) < 1e-12
+        assert 1 - N * (r["max_left"][b] + K * tol) - 1e-9 <= r["sum_lambda"][b] <= 1 + 1e-9
+        # the paper reports up to 50 matchings and coefficients of a few hundredths for an 8 x 8 matrix
+        # (Sec. 4.2): same order of magnitude here (mean coefficient = about 1 / K)
+        assert 0.01 < r["sum_lambda"][b] / K < 0.1 and 3 * N < K <= 50
+
+
+def test_real_bvn_stops_without_a_perfect_matching_and_rejects_bad_entries():
+    A = np.array([[[0.5, 0.5, 0.0], [0.5, 0.5, 0.0], [0.0, 0.0, 0.0]]])
+    r = oracle.bvn_real_decompose(A, 10)
+    assert r["count"][0] == 0 and r["status"][0] == 1 and r["max_left"][0] == 0.5
+    A = np.array([[[0.5, 0.5], [0.5, 0.25]]])                         # the second matching exhausts row 1 early
+    r = oracle.bvn_real_decompose(A, 10, tol=0.0)
+    assert r["count"][0] == 2 and list(r["lam"][0, :2]) == [0.25, 0.5] and r["status"][0] == 1
+    assert r["max_left"][0] == 0.25 and r["sum_lambda"][0] == 0.75
+    A = np.array([[[0.5, -0.1], [0.5, 0.5]], [[np.nan, 0.1], [0.5, 0.5]]])
+    r = oracle.bvn_real_decompose(A, 10)
+    assert list(r["status"]) == [-1, -1] and (r["count"] == 0).all()
+    r = oracle.bvn_real_decompose(np.array([[[1.0, 1e-13], [1e-13, 1.0]]]), 10, tol=1e-12)
+    assert r["count"][0] == 1 and r["status"][0] == 0               # entries at the tolerance count as zero
+    r = oracle.bvn_real_decompose(np.full((1, 4, 4), 0.25), 2, tol=0.0)
+    assert r["count"][0] == 2 and r["status"][0] == 1               # budget reached with entries left
