@@ -345,6 +345,31 @@ int moesched_sinkhorn_durations(int B, int k_stride, const int32_t* d_coef, cons
                                 const double* d_stretch, int scale_bits, int32_t* d_dur, void* stream);
 
 /*
+ * Birkhoff-von Neumann decomposition of a real-valued matrix (paper Sec. 3.1: A = sum_k lambda_k P_k
+ * for a doubly stochastic A; Sec. 4.2 discusses the size of its coefficients). The usual input is
+ * d_scaled of moesched_sinkhorn_scale, which is doubly stochastic only up to the error of its last
+ * sweep; so entries at or below `tol` count as zero (on input and after every subtraction) and the
+ * loop also ends when the support has no perfect matching left. Per step: pi_k = lexicographically
+ * smallest permutation with positive entries, lambda_k = its smallest entry, subtracted along pi_k.
+ * Single IEEE double operations in a fixed order: results are reproducible bit for bit.
+ *
+ *   d_matrix     in   [B][N][N] double, entries >= 0 (a negative or NaN entry: BAD_INPUT)
+ *   tol          in   >= 0
+ *   k_max        in   output capacity, >= 1 (N^2 - 2N + 2 always suffices)
+ *   d_perm       out  [B][k_max][N] uint8
+ *   d_lambda     out  [B][k_max] double coefficients
+ *   d_count      out  [B] int32
+ *   d_sum_lambda out  [B] double: ((lambda_0 + lambda_1) + ...), 1 up to what is left for a scaled matrix
+ *   d_max_left   out  [B] double: the largest entry remaining when the loop ended
+ *   d_scratch    tmp  B * N * roundup(N, 8) doubles, 8-byte aligned: the working copy
+ *   d_status     out  [B] int32: OK (nothing left), TRUNCATED (entries left: no perfect matching any
+ *                     more, or k_max reached), BAD_INPUT (count 0)
+ */
+int moesched_bvn_real_decompose(int B, int N, const double* d_matrix, double tol, int k_max, uint8_t* d_perm,
+                                double* d_lambda, int32_t* d_count, double* d_sum_lambda, double* d_max_left,
+                                double* d_scratch, int32_t* d_status, void* stream);
+
+/*
  * Birkhoff-von Neumann decomposition for callers that cannot allocate device memory.
  * (The paper has no counterpart: this is a packaging variant of moesched_bvn_decompose,
  * same arguments, same results, minus d_scratch.)

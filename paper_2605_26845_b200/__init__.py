@@ -51,7 +51,8 @@ def load_library():
         for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
                      "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
                      "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error",
-                     "moesched_schedule_order", "moesched_schedule_permute", "moesched_best_budget"):
+                     "moesched_schedule_order", "moesched_schedule_permute", "moesched_best_budget",
+                     "moesched_bvn_real_decompose"):
             getattr(lib, name).restype = ctypes.c_int
         lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
         lib.moesched_order_scratch_bytes.restype = ctypes.c_size_t
@@ -251,6 +252,32 @@ def sinkhorn_durations(coef, count, stretch, scale_bits=20, out=None) -> torch.T
     rc = load_library().moesched_sinkhorn_durations(B, K, _ptr(coef), _ptr(count), _ptr(stretch), int(scale_bits),
                                                     _ptr(_dev(out, torch.int32, "out")), _stream(coef.device))
     _check(rc, "moesched_sinkhorn_durations")
+    return out
+
+
+def bvn_real_decompose(matrix, k_max=None, tol=1e-12) -> dict:
+    """Real-valued Birkhoff-von Neumann decomposition A = sum_k lambda_k P_k (paper Sec. 3.1) of [B, N, N]
+    float64 matrices, e.g. sinkhorn_scale(...)["scaled"]. Returns perm [B, k_max, N] uint8, lam [B, k_max]
+    float64, count, sum_lambda, max_left (largest entry remaining) and status [B]."""
+    lib = load_library()
+    matrix = _dev(matrix, torch.float64, "matrix")
+    if matrix.dim() != 3 or matrix.shape[1] != matrix.shape[2]:
+        raise MoeschedError("matrix must have shape [B, N, N]")
+    B, N, _ = matrix.shape
+    dev = matrix.device
+    k_max = bvn_capacity(N) if k_max is None else int(k_max)
+    out = dict(perm=torch.empty((B, k_max, N), dtype=torch.uint8, device=dev),
+               lam=torch.empty((B, k_max), dtype=torch.float64, device=dev),
+               count=torch.empty(B, dtype=torch.int32, device=dev),
+               sum_lambda=torch.empty(B, dtype=torch.float64, device=dev),
+               max_left=torch.empty(B, dtype=torch.float64, device=dev),
+               status=torch.empty(B, dtype=torch.int32, device=dev))
+    scratch = torch.empty(max(1, B * N * ((N + 7) // 8 * 8)), dtype=torch.float64, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib.moesched_bvn_real_decompose(B, N, _ptr(matrix), ctypes.c_double(float(tol)), k_max, _ptr(out["perm"]),
+                                             _ptr(out["lam"]), _ptr(out["count"]), _ptr(out["sum_lambda"]),
+                                             _ptr(out["max_left"]), _ptr(scratch), _ptr(out["status"]), _stream(dev))
+    _check(rc, "moesched_bvn_real_decompose")
     return out
 
 

@@ -7,7 +7,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["api.cu", "mw_kernel.cu", "mw_team_kernel.cu", "bvn_kernel.cu", "bvn_team_kernel.cu", "eval_kernel.cu", "eval_team_kernel.cu", "order_kernel.cu", "bvn_static.cu", "probe.cu", "a2a_kernel.cu", "sinkhorn_kernel.cu"]
+SOURCES = ["api.cu", "mw_kernel.cu", "mw_team_kernel.cu", "bvn_kernel.cu", "bvn_team_kernel.cu", "bvn_real_kernel.cu", "eval_kernel.cu", "eval_team_kernel.cu", "order_kernel.cu", "bvn_static.cu", "probe.cu", "a2a_kernel.cu", "sinkhorn_kernel.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "team.cuh"), os.path.join(HERE, "..", "include", "moesched.h")]
 LIB = os.path.join(HERE, "libmoesched.so")
 

@@ -252,6 +252,21 @@ int moesched_sinkhorn_durations(int B, int k_stride, const int32_t* d_coef, cons
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
 }
 
+int moesched_bvn_real_decompose(int B, int N, const double* d_matrix, double tol, int k_max, uint8_t* d_perm,
+                                double* d_lambda, int32_t* d_count, double* d_sum_lambda, double* d_max_left,
+                                double* d_scratch, int32_t* d_status, void* stream) {
+  if (B < 0 || N < 1 || N > MOESCHED_MAX_N || k_max < 1 || !(tol >= 0.0)) return MOESCHED_EINVAL;
+  if (B == 0) return MOESCHED_OK;
+  if (!d_matrix || !d_perm || !d_lambda || !d_count || !d_sum_lambda || !d_max_left || !d_scratch || !d_status)
+    return MOESCHED_EINVAL;
+  if (!aligned8(d_matrix) || !aligned8(d_lambda) || !aligned8(d_sum_lambda) || !aligned8(d_max_left) ||
+      !aligned8(d_scratch) || !aligned4(d_count) || !aligned4(d_status))
+    return MOESCHED_EINVAL;
+  cudaError_t e = run_bvn_real(B, N, d_matrix, tol, k_max, d_perm, d_lambda, d_count, d_sum_lambda, d_max_left,
+                               d_scratch, d_status, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
 int moesched_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* moesched_strerror(int code) {

@@ -1028,6 +1028,10 @@ cudaError_t run_sinkhorn(int B, int N, const int32_t* demand, int iters, double 
 cudaError_t run_sinkhorn_durations(int B, int k_stride, const int32_t* coef, const int32_t* count,
                                    const double* stretch, int scale_bits, int32_t* dur, cudaStream_t stream);
 
+cudaError_t run_bvn_real(int B, int N, const double* matrix, double tol, int k_max, uint8_t* perm, double* lambda,
+                         int32_t* count, double* sum_lambda, double* max_left, double* scratch, int32_t* status,
+                         cudaStream_t stream);
+
 // Launch helper shared by the three kernels.
 template <typename Kernel, typename... Args>
 cudaError_t launch_warp_kernel(Kernel kern, const Geometry& ge, int B, cudaStream_t stream, Args... args) {

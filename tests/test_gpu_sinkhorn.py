@@ -119,3 +119,58 @@ def test_full_size_headline_batch_properties():
     r = oracle.sinkhorn_scale(D[sample], 20, 0.5, 20, threads=8)
     assert (S[sample] == r["scaled"]).all() and (Q[sample] == r["fixed"]).all()
     assert (g["stretch"].cpu().numpy()[sample] == r["stretch"]).all()
+
+
+# ---- real-valued Birkhoff-von Neumann decomposition of the scaled matrix (paper Sec. 3.1) ----
+
+def assert_real_bvn_equal(A, k_max, tol, threads=8):
+    g = ms.bvn_real_decompose(dev(A), k_max, tol)
+    r = oracle.bvn_real_decompose(A, k_max, tol=tol, threads=threads)
+    count = g["count"].cpu().numpy()
+    assert (g["status"].cpu().numpy() == r["status"]).all() and (count == r["count"]).all()
+    kk = np.arange(k_max)[None, :] < count[:, None]
+    assert (g["perm"].cpu().numpy()[kk] == r["perm"][kk]).all()
+    assert (g["lam"].cpu().numpy()[kk] == r["lam"][kk]).all()                  # doubles, bit for bit
+    assert (g["sum_lambda"].cpu().numpy() == r["sum_lambda"]).all()
+    assert (g["max_left"].cpu().numpy() == r["max_left"]).all()
+    return g, r
+
+
+@pytest.mark.parametrize("N", [1, 2, 5, 8, 17, 32, 33, 64, 100, 129, 200])
+def test_real_bvn_of_scaled_matrices_is_bit_identical_to_the_oracle(N):
+    B = 6 if N <= 64 else 2
+    D = random_matrices(B, N, seed=500 + N, kind="uniform", high=300, zero_frac=0.4)
+    sk = oracle.sinkhorn_scale(D, 60, 0.5, 20, threads=8)
+    k_max = bvn_capacity(N) if N <= 64 else 150
+    g, r = assert_real_bvn_equal(sk["scaled"], k_max, 1e-9)
+    if N <= 64:
+        assert (np.abs(r["sum_lambda"] - 1.0) < 1e-3).all()                    # the coefficients add up to one
+
+
+def test_real_bvn_of_the_workload_and_special_inputs():
+    D = make_demand(3, 24)
+    sk = oracle.sinkhorn_scale(D, 20, 0.5, 20, threads=8)
+    g, r = assert_real_bvn_equal(sk["scaled"], bvn_capacity(64), 1e-9)
+    assert (r["count"] > 500).all()                                           # thousands of small matchings
+    # exact inputs, early end without a perfect matching, rejected entries, a short budget
+    N = 8
+    A = np.zeros((7, N, N))
+    A[0] = 1.0 / N
+    A[1, np.arange(N), np.roll(np.arange(N), 3)] = 1.0
+    A[2, :2, :2] = 0.5                                                         # no perfect matching at all
+    A[3] = 1.0 / N
+    A[3, 4, 4] = -0.25
+    A[4] = 1.0 / N
+    A[4, 1, 1] = np.nan
+    A[5] = random_matrices(1, N, seed=9, kind="uniform", high=64)[0] / 64.0   # not balanced: stops early
+    A[6] = 1e-13                                                               # everything below the tolerance
+    g, r = assert_real_bvn_equal(A, 20, 1e-12)
+    assert list(r["status"]) == [0, 0, 1, -1, -1, 1, 0] and r["count"][0] == N and r["count"][6] == 0
+    assert_real_bvn_equal(A[:1], 3, 0.0)                                       # budget reached: TRUNCATED
+    # dyadic matrices: the integer decomposition, scaled (see the oracle's pin), on the GPU as well
+    D = random_matrices(4, 16, seed=3, kind="uniform", high=40, zero_frac=0.4)
+    v = ms.bvn_decompose(dev(D), want_aug=True)
+    g = ms.bvn_real_decompose(v.extra.double() / 4096.0, tol=0.0)
+    assert (g["count"] == v.count).all() and (g["status"] == 0).all()
+    kk = torch.arange(g["perm"].shape[1], device="cuda")[None, :] < v.count[:, None]
+    assert (g["perm"][kk] == v.perm[kk]).all() and (g["lam"][kk] == v.dur[kk].double() / 4096.0).all()
