@@ -195,7 +195,9 @@ size_t moesched_workspace_bytes(int B, int N, int k_max);
  *   d_demand  in   [B][N][N] int32, entries >= 0
  *   k_stride  in   matchings allocated per matrix in d_perm / d_dur
  *   d_perm    in   [B][k_stride][N] uint8, each used row a permutation of 0..N-1
- *   d_dur     in   [B][k_stride] int32, >= 0, sum over k <= 2^40
+ *   d_dur     in   [B][k_stride] int32, >= 0, sum over k <= 2^40; the dispatch stage
+ *                  (sum of reconfig_ns + t_k) and the expert batches (sum of comp_k) must each
+ *                  stay within 2^60 ns, so that no makespan can wrap (BAD_INPUT otherwise)
  *   d_count   in   [B] int32, 0 <= count <= k_stride
  *   h_model   in   HOST pointer, read during the call
  *   d_*       out  [B] int64 each; zero when status is BAD_INPUT

@@ -403,6 +403,10 @@ i64 batch_time(const Model& m, i64 g) {
 }
 
 const i64 DUR_SUM_MAX = 1LL << 40;
+// Input range of the scoring: the summed stage times must stay clear of 63 bits. A schedule whose
+// dispatch stage (sum of reconfiguration + transfer times) or whose expert batches add up to more than
+// 2^60 ns is rejected, so that no makespan can wrap silently.
+const i64 STAGE_SUM_MAX = 1LL << 60;
 
 void eval_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t* dur,
               const Model& m, i64* overlap, i64* serial, i64* idle_ns, i64* idle_tok,
@@ -423,7 +427,7 @@ void eval_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t
   }
   if (dsum > DUR_SUM_MAX) { *status = ST_BAD_INPUT; return; }
   std::vector<i64> R(D, D + NN);
-  i64 dsp = 0, cmp = 0, cmb = 0, ser = 0, comp_sum = 0, idle_t = 0, dsp1 = 0;
+  i64 dsp = 0, cmp = 0, cmb = 0, ser = 0, comp_sum = 0, idle_t = 0, dsp1 = 0, leg_sum = 0;
   for (int k = 0; k < K; ++k) {
     i64 g = 0, s = 0;
     for (int i = 0; i < N; ++i) {
@@ -443,6 +447,8 @@ void eval_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_t
     cmb = std::max(cmp, cmb) + m.reconfig_ns + t;  // results return over the same pairs
     ser += 2 * (m.reconfig_ns + t) + comp;
     comp_sum += comp;
+    leg_sum += m.reconfig_ns + t;
+    if (leg_sum > STAGE_SUM_MAX || comp_sum > STAGE_SUM_MAX) { *status = ST_BAD_INPUT; return; }
     idle_t += (i64)N * dur[k] - s;
   }
   *overlap = cmb;

@@ -741,6 +741,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       }
     }
     int level = 0;
+    work[WK_POP]++;   // row i itself
     hist_store<W>(hist, 0, F, lane);
     for (int it = 0; it < N; ++it) {
       unsigned acc[W];
@@ -765,6 +766,8 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       work[WK_LEVEL]++;
       if (!grew) break;
       ++level;
+#pragma unroll
+      for (int w = 0; w < W; ++w) work[WK_POP] += __popc(F[w]);
       hist_store<W>(hist, level, F, lane);
     }
     __syncwarp();

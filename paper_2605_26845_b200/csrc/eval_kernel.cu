@@ -183,6 +183,8 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
       ser += warp_sum64(2 * leg_mine + comp_mine);
       comp_sum += warp_sum64(comp_mine);
       dur_sum += warp_sum64((long long)dk_mine);
+      // stage sums beyond 2^60 ns are out of range (a chunk adds less than 2^61, so nothing has wrapped yet)
+      if (ser - comp_sum > (2LL << 60) || comp_sum > (1LL << 60)) { bad = 1; break; }
       long long cmb_mine = 0;
       for (int q = 0; q < kend; ++q) {
         const long long leg = __shfl_sync(FULL, leg_mine, q);
@@ -280,7 +282,7 @@ cudaError_t run_eval(int B, int N, const int32_t* demand, int k_stride, const ui
     // as in the greedy path: narrow matrices first, in the 16-bit layout, then the rest
     cudaError_t e = classify_matrices(B, N, demand, status, stream);
     if (e != cudaSuccess) return e;
-    if (N > 128 && B < 8 * sm_count() && prefix_overlap == nullptr) {
+    if (N > 128 && B < 8 * sm_count() && prefix_overlap == nullptr && k_stride <= 65535 * 32) {
       // few large matrices: one CTA per matrix instead of one warp (N = 256, B = 256 on a BvN schedule:
       // 33 ms against 74 ms; at N = 128, B = 1024 one warp per matrix is the faster, 17 ms against 20 ms)
       e = run_eval_team(B, N, demand, k_stride, perm, dur, count, model, overlap, serial, idle_ns, idle_tok, unserved,

@@ -15,7 +15,7 @@ namespace {
 struct EvalTeamState {
   int gmax[32];        // largest served pair of each matching of the chunk
   int dur[32];         // its duration
-  int flags[4];        // 0: chunk is bad
+  int flags[4];        // 0: chunk is bad, 1: a sum left its range
   long long sums[4];   // block reductions: total demand, leftover
 };
 
@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(32 * NW) eval_team_kernel(int B, int N, const 
 
   for (int k0 = 0, chunk = 1; !bad && k0 < K; k0 += 32, ++chunk) {
     const int kend = min(32, K - k0);
-    const unsigned short stamp = (unsigned short)chunk;   // at most 2033 chunks: never 0, never repeats
+    const unsigned short stamp = (unsigned short)chunk;   // the launcher admits at most 65535 chunks: never 0, never repeats
     if (t < 32) {
       const int dk = t < kend ? db[k0 + t] : 0;
       st->dur[t] = dk;
@@ -143,6 +143,8 @@ __global__ void __launch_bounds__(32 * NW) eval_team_kernel(int B, int N, const 
       ser += a;
       comp_sum += c;
       dur_sum += d;
+      // stage sums beyond 2^60 ns are out of range (a chunk adds less than 2^61, so nothing has wrapped yet)
+      if (lane == 0 && (ser - comp_sum > (2LL << 60) || comp_sum > (1LL << 60))) st->flags[1] = 1;
       for (int q = 0; q < kend; ++q) {
         const long long leg = __shfl_sync(FULL, leg_mine, q);
         const long long comp = __shfl_sync(FULL, comp_mine, q);
@@ -153,6 +155,7 @@ __global__ void __launch_bounds__(32 * NW) eval_team_kernel(int B, int N, const 
       }
     }
     __syncthreads();
+    if (st->flags[1]) { bad = true; break; }
   }
   if (warp == 0 && lane == 0 && dur_sum > (1LL << 40)) st->flags[1] = 1;
   __syncthreads();

@@ -213,7 +213,7 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
     if (ikey == 0xffffffffu) break;
     const int i = (int)(ikey >> 16);
     from = i + 1;
-    if (t == 0) work[WK_SWEEP]++;
+    if (t == 0) { work[WK_SWEEP]++; work[WK_POP]++; }
     // Every search takes a fresh range of N + 2 level stamps, so that the marks of earlier searches
     // never need clearing. Before the stamps could pass 2^31 (after some 8 million searches at
     // N = 256; a complete worst-case decomposition can get there) all marks are wiped and the
@@ -249,7 +249,11 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
       red.close();
       red.read_set<W>(xf);
       red.next();
-      if (t == 0) work[WK_LEVEL]++;
+      if (t == 0) {
+        work[WK_LEVEL]++;
+#pragma unroll
+        for (int w = 0; w < W; ++w) work[WK_POP] += __popc(xf[w]);
+      }
       if (!any_bit<W>(xf)) break;
       ++level;
     }
@@ -474,6 +478,11 @@ __device__ __forceinline__ int warp_rotate(TeamShared<NW>& sh, const TeamSearchS
 // Lexicographically smallest perfect matching of the graph (ts.cc / ts.rr, m.Rr) over the rows
 // [start, N), given a perfect matching that already equals the answer below `start`; see
 // canonicalise() in common.cuh for the argument. Same result as team_canonicalise. Uniform.
+// (For the Birkhoff kernel, whose windows hold one to three rows that could move, this scheme, with
+// the search records added, was measured slower than team_canonicalise: 1.85 s against 1.06 s on 256
+// matrices of 256 ranks. With nothing to search side by side, one warp working while seven wait is
+// worse than eight warps sharing every level. It serves the greedy kernel, where every step
+// searches the whole matrix.)
 template <int NW>
 __device__ __forceinline__ bool team_canonicalise_par(TeamShared<NW>& sh, TeamSearchShared<NW>& ts, TeamRed& red, int N,
                                                       int t, int lane, int warp, bool in, TeamMatch<NW>& m, int& stamp,

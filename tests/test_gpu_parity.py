@@ -220,6 +220,27 @@ def test_large_matrix_scoring_rejects_bad_schedules_and_scores_long_ones(N):
             assert (s[name].cpu().numpy() == r[name]).all(), name
 
 
+@pytest.mark.parametrize("N", [4, 64, 200])
+def test_stage_sums_out_of_range_are_rejected_like_the_oracle_does(N):
+    """Slowest link, largest token: transfer times that add up beyond 2^60 ns give BAD_INPUT, not a wrapped
+    makespan; just below the limit the 64-bit sums are still exact (one-warp and CTA-per-matrix kernels)."""
+    K = 600
+    D = random_matrices(3, N, seed=31 + N, kind="uniform", high=100)
+    perm = np.tile(np.arange(N, dtype=np.uint8), (3, K, 1))
+    dur = np.zeros((3, K), np.int32)
+    dur[0, :128] = 2**31 - 1
+    dur[1, :32] = 2**31 - 1
+    dur[2, 500:] = 2**31 - 1                       # the sum leaves its range late in the schedule
+    count = np.array([K, K, K], np.int32)
+    model = dict(DEFAULT_MODEL, bytes_per_token=2**20, link_gbps=1)
+    for prefix in (False, True):
+        s = ms.schedule_eval(dev(D), dev(perm), dev(dur), dev(count), model, prefix=prefix)
+        r = oracle.schedule_eval(D, perm, dur, count, model)
+        assert list(r["status"]) == [-1, 0, -1]
+        for name in ms.SCORE_FIELDS + ("status",):
+            assert (s[name].cpu().numpy() == r[name]).all(), name
+
+
 def test_argument_errors_are_reported():
     d = dev(make_demand(1, 2))
     with pytest.raises(ms.MoeschedError):

@@ -250,3 +250,22 @@ def test_prefix_scores_are_the_scores_of_the_truncated_schedules():
     perm[0, 1] = [1, 1]
     bad = oracle.schedule_prefix_eval(D, perm, dur, np.array([3], np.int32), model)
     assert bad["status"][0] == -1 and (bad["prefix_overlap_ns"] == -1).all()
+
+
+def test_stage_sums_beyond_2_to_60_ns_are_rejected_not_wrapped():
+    """With the slowest link and the largest token the summed transfer times can pass 63 bits; the
+    scoring rejects a schedule whose dispatch stage exceeds 2^60 ns instead of returning a wrapped sum."""
+    N, K = 4, 600
+    D = np.zeros((2, N, N), np.int32)
+    perm = np.tile(np.arange(N, dtype=np.uint8), (2, K, 1))
+    dur = np.zeros((2, K), np.int32)
+    dur[0, :128] = 2**31 - 1            # sum 2^38: transfer times add up to about 2^61 ns at 2^23 ns per token
+    dur[1, :32] = 2**31 - 1             # sum 2^36: about 2^59 ns, within range
+    count = np.array([K, K], np.int32)
+    model = dict(DEFAULT_MODEL, bytes_per_token=2**20, link_gbps=1)
+    r = oracle.schedule_eval(D, perm, dur, count, model)
+    assert list(r["status"]) == [-1, 0]
+    assert r["makespan_overlap_ns"][0] == 0 and r["makespan_serial_ns"][0] == 0
+    t = (2**31 - 1) * 2**23
+    assert r["makespan_serial_ns"][1] == 2 * (32 * t + K * model["reconfig_ns"])
+    assert r["makespan_overlap_ns"][1] > 2**59
