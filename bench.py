@@ -137,14 +137,38 @@ def captured_traffic(name):
 
 
 def algorithmic_ops(work_mw, work_bvn, N):
-    """Integer lane-operations the method itself needs, from the kernels' work counters
-    (per column or row touched: a handful of adds / compares / bit operations)."""
+    """Integer lane-operations of the DATA-PARALLEL formulation the kernels run, from their work counters:
+    a search level is taken by all lanes over all mask words (4 N W), a column scan costs 6 N, and so on.
+    This counts what a lane-parallel machine has to issue for the method, not what a scalar one would."""
     W = (N + 31) // 32
     mw = (6 * N * work_mw[:, 0] + 4 * work_mw[:, 1] + 4 * N * work_mw[:, 2] + 4 * N * W * work_mw[:, 4]
           + 6 * N * work_mw[:, 5] + 4 * N * work_mw[:, 6] + 4 * N * work_mw[:, 3])
     bvn = (4 * N * W * work_bvn[:, 0] + 4 * work_bvn[:, 1] + 4 * N * W * work_bvn[:, 4] + 6 * N * work_bvn[:, 5]
            + 6 * N * work_bvn[:, 6] + 4 * N * work_bvn[:, 3])
     return float(mw.sum()), float(bvn.sum())
+
+
+def scalar_model_ops(work_mw, work_bvn, N):
+    """Integer operations of the method itself under the scalar cost model: per scanned column an add
+    pair, a min-update and a compare-select (4 N per scan S), 2 N per dual update U, N/32 word
+    operations per frontier row L popped by a canonicalisation search, 3 N per matching K for serve
+    and emit; Birkhoff: 2 N per augmenting-path step, the same search and emit terms, 4 N^2 once for
+    the sums and the padding. Counters: greedy S = field 0, U = field 1 (one dual update per
+    augmentation), L = field 8, K = field 6; Birkhoff path steps = field 1, L = field 8, K = field 6."""
+    mw = 4 * N * work_mw[:, 0] + 2 * N * work_mw[:, 1] + (N / 32) * work_mw[:, 8] + 3 * N * work_mw[:, 6]
+    bvn = 2 * N * work_bvn[:, 1] + (N / 32) * work_bvn[:, 8] + 3 * N * work_bvn[:, 6] + 4 * N * N
+    return float(mw.sum()), float(bvn.sum())
+
+
+WORK_NAMES_MW = ("column_scans", "augmentations", "rows_bid", "searches", "search_levels", "rotation_steps",
+                 "matchings", "rows_matched_on_tight_edges", "frontier_pops", "settled_groups")
+WORK_NAMES_BVN = ("repair_levels", "repair_path_steps", "unused", "searches", "search_levels", "rotation_steps",
+                  "matchings", "rows_skipped_as_prefix", "frontier_pops", "unused")
+
+
+def per_matching(work, names):
+    k = max(1.0, float(work[:, 6].sum()))
+    return {n: float(work[:, i].sum()) / k for i, n in enumerate(names) if n not in ("unused", "matchings")}
 
 
 def rank_demand(rank, B):
@@ -220,6 +244,8 @@ def main():
                     help="replay the step from a CUDA graph (pays off when the kernels take microseconds)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="keep greedy and BvN on one stream instead of forking them onto two")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also time the greedy decomposition at every budget of the configuration (rates_by_k_max)")
     ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS),
                     help="workload configuration (default 3: N=64, the one the metric is quoted on)")
     args = ap.parse_args()
@@ -347,6 +373,52 @@ def main():
     sk_ok = bool((sk["status"] == 0).all())
     del sk
 
+    # ---- order of the matchings (not part of the step): best of five orders of the greedy schedule ----
+    compute_bound = dict(DEFAULT_MODEL, expert_ps_per_token=400_000)     # an expert token costs more than its transfer
+    ordering = {}
+    if K_MW <= ms.ORDER_MAX_K:
+        fixed_list = cfg.get("expert_fixed_ns", (DEFAULT_MODEL["expert_fixed_ns"],))
+        models = [("fixed_%dus" % (f // 1000), dict(DEFAULT_MODEL, expert_fixed_ns=f)) for f in fixed_list]
+        models.append(("compute_bound_400ns_per_token", compute_bound))
+        for name, model in models:
+            ms.schedule_order(d, mw.perm, mw.dur, mw.count, model)          # allocations and first-use set-up
+            flush.fill_(1)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            od = ms.schedule_order(d, mw.perm, mw.dur, mw.count, model)
+            a1.record(stream)
+            a1.synchronize()
+            gain = ((od["emission_ns"] - od["makespan_ns"]).double() / od["emission_ns"].double().clamp(min=1)).mean()
+            ordering[name] = {"ms": a0.elapsed_time(a1), "mean_makespan_gain_frac": float(gain),
+                              "schedules_reordered_frac": float((od["rule"] != 0).double().mean())}
+
+    # ---- greedy at every budget of the configuration (--sweep), scored ----
+    rates_by_k = {}
+    if args.sweep:
+        for kb in cfg["k_max"]:
+            sch = ms._new_schedule(d, kb, False, False)
+            ts = []
+            for _ in range(3):
+                flush.fill_(1)
+                a0, a1, a2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                a0.record(stream)
+                ms.mw_decompose(d, kb, out=sch)
+                a1.record(stream)
+                sc = ms.schedule_eval(d, sch.perm, sch.dur, sch.count, DEFAULT_MODEL)
+                a2.record(stream)
+                a2.synchronize()
+                ts.append((a0.elapsed_time(a1), a1.elapsed_time(a2)))
+            t_mw, t_ev = (float(np.median([t[i] for t in ts])) for i in (0, 1))
+            entry = {"greedy_ms": t_mw, "scoring_ms": t_ev, "greedy_per_s": B / (t_mw * 1e-3),
+                     "mean_unserved_frac": float((sc["unserved_tokens"].double() / d.sum((1, 2)).double()).mean()),
+                     "mean_makespan_overlap_us": float(sc["makespan_overlap_ns"].double().mean()) / 1e3}
+            for f in cfg.get("expert_fixed_ns", ()):
+                sf = ms.schedule_eval(d, sch.perm, sch.dur, sch.count, dict(DEFAULT_MODEL, expert_fixed_ns=f))
+                entry["mean_makespan_overlap_us_fixed_%dus" % (f // 1000)] = \
+                    float(sf["makespan_overlap_ns"].double().mean()) / 1e3
+            rates_by_k[str(kb)] = entry
+            del sch
+
     # ---- end to end: pinned host demand in, schedules and scores back to pinned host memory, every step;
     # the public double-buffered runner overlaps one step's copies with the next step's kernels ----
     h_in = torch.from_numpy(D_host).pin_memory()
@@ -386,11 +458,17 @@ def main():
         peaks, peak_kind = measured_peaks()
         sm_mhz = ck["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
         ops_mw, ops_bvn = algorithmic_ops(work_mw, work_bv, N)
+        sc_mw, sc_bvn = scalar_model_ops(work_mw, work_bv, N)
         dom = int(np.argmax(per_kernel))
         dom_ops = ops_bvn if dom == 2 else ops_mw
+        dom_scalar = sc_bvn if dom == 2 else sc_mw
         alu_peak = ALU_LANES_PER_CLK * sm_mhz * 1e6 / 1e9          # G lane-ops/s at the sampled clock
         alu_measured = ms.probe_int_rate(dev) / 1e9                 # add / min / logic mix, measured now
-        achieved = dom_ops / (per_kernel[dom] * 1e-3) / 1e9
+        achieved_par = dom_ops / (per_kernel[dom] * 1e-3) / 1e9
+        achieved = dom_scalar / (per_kernel[dom] * 1e-3) / 1e9
+        other = 0 if dom == 2 else 2
+        other_scalar = sc_mw if dom == 2 else sc_bvn
+        other_par = ops_mw if dom == 2 else ops_bvn
         k_bv = float(bv.count.double().mean())
         k_mw = float(mw.count.double().mean())
         bytes_bvn = B * (4 * N * N + k_bv * (N + 4) + 8)
@@ -406,10 +484,35 @@ def main():
             "kernels_ms": {n: float(t) for n, t in zip(names, per_kernel)},
             "kernels_ms_note": "per-kernel events from a second, identical serial pass",
             "rates": {"greedy_per_s": B / (per_kernel[0] * 1e-3), "bvn_per_s": B / (per_kernel[2] * 1e-3)},
+            # frac: the method's own integer operations (scalar cost model, see scalar_model_ops) over the
+            # issue-rate peak; frac_parallel_formulation: the lane-operations of the data-parallel formulation
+            # (algorithmic_ops: a search level costs all lanes over all mask words, whether or not a lane's
+            # rows are in the frontier) over the same peak. Both can be recomputed from work_per_matching.
             "roofline": {"kernel": names[dom], "bound": "alu", "achieved": achieved, "peak": alu_peak,
-                         "unit": "Gop/s", "frac": achieved / alu_peak, "traffic": captured_traffic(names[dom]) if CFG == 3 else None,
+                         "unit": "Gop/s", "frac": achieved / alu_peak,
+                         "ops_per_launch": dom_scalar, "ops_model": "scalar: 4NS+2NU+(N/32)L+3NK (greedy), "
+                         "2N*path_steps+(N/32)L+3NK+4N^2 (BvN)",
+                         "frac_parallel_formulation": achieved_par / alu_peak,
+                         "ops_per_launch_parallel_formulation": dom_ops,
+                         "traffic": captured_traffic(names[dom]) if CFG == 3 else None,
                          "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (sampled)",
                          "peak_measured_int_mix": alu_measured, "frac_of_measured_int_mix": achieved / alu_measured,
+                         "frac_parallel_formulation_of_measured_int_mix": achieved_par / alu_measured,
+                         "work_per_matching": {"greedy": per_matching(work_mw, WORK_NAMES_MW),
+                                               "bvn": per_matching(work_bv, WORK_NAMES_BVN)},
+                         "other_decomposer": {"kernel": names[other],
+                                              "frac": other_scalar / (per_kernel[other] * 1e-3) / 1e9 / alu_peak,
+                                              "frac_parallel_formulation":
+                                                  other_par / (per_kernel[other] * 1e-3) / 1e9 / alu_peak,
+                                              "ops_per_launch": other_scalar},
+                         "scoring_kernel_hbm": {"kernel": names[3], "bound": "hbm",
+                                                "algorithmic_bytes": B * (4 * N * N + k_bv * (N + 4) + 48),
+                                                "achieved_gbs": B * (4 * N * N + k_bv * (N + 4) + 48)
+                                                / (per_kernel[3] * 1e-3) / 1e9,
+                                                "frac": B * (4 * N * N + k_bv * (N + 4) + 48)
+                                                / (per_kernel[3] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                "traffic": captured_traffic(names[3]) if CFG == 3 else None,
+                                                "peak_kind": f"of {peak_kind}"},
                          "hbm_side": {"algorithmic_bytes": bytes_bvn,
                                       "gbs": bytes_bvn / (per_kernel[2] * 1e-3) / 1e9,
                                       "peak_gbs": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}"}},
@@ -423,6 +526,7 @@ def main():
                                 "achieved": 16.0 * B * N * N / (sk_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                 "unit": "GB/s", "frac": 16.0 * B * N * N / (sk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                 "peak_kind": f"of {peak_kind}", "all_status_ok": sk_ok},
+            "ordering": ordering,
             "e2e": {"value": aggregate_value(world, B, e2e_steps, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "how": "HostPipeline: upload, kernels and download on three streams, two slots",
@@ -432,6 +536,8 @@ def main():
             "gpu_launches": (4 if N < 48 else 10) * args.steps,
             "clocks": ck,
         }
+        if rates_by_k:
+            out["rates_by_k_max"] = rates_by_k
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
