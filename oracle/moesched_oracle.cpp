@@ -103,50 +103,68 @@ bool t0_support_perm(int N, const i64* A, int* perm) {
 }
 
 // ---------------------------------------------------------------------------
-// Assignment problem: maximum total weight over permutations, textbook
-// shortest-augmenting-path method with potentials on cost = -weight.
-// Returns the optimum; fills row->column assignment and the duals (of the
-// cost problem: pu[i] + pv[j] <= cost[i][j], equality on matched edges).
+// Assignment problem: maximum total weight over permutations, by successive
+// shortest augmenting paths on cost = -weight with row and column potentials.
+// Rows are inserted one at a time: a shortest-path tree over the reduced costs
+// cost[i][j] - pu[i] - pv[j] (all >= 0) is grown from the new row until it
+// reaches a free column; the potentials are then moved so that every edge of
+// the tree stays tight and the path is flipped. Returns the optimum; fills the
+// row -> column assignment and the duals (of the cost problem:
+// pu[i] + pv[j] <= cost[i][j], equality on matched edges).
 // ---------------------------------------------------------------------------
-i64 assignment_max(int N, const i64* W, int* row_to_col, i64* pu, i64* pv) {
+i64 assignment_max(int N, const i64* W, int* row_to_col, i64* pu_out, i64* pv_out) {
   const i64 INF = std::numeric_limits<i64>::max() / 4;
-  std::vector<i64> u(N + 1, 0), v(N + 1, 0), minv(N + 1);
-  std::vector<int> p(N + 1, 0), way(N + 1, 0);
-  std::vector<char> used(N + 1);
-  for (int i = 1; i <= N; ++i) {
-    p[0] = i;
-    int j0 = 0;
-    std::fill(minv.begin(), minv.end(), INF);
-    std::fill(used.begin(), used.end(), 0);
-    do {
-      used[j0] = 1;
-      int i0 = p[j0], j1 = 0;
-      i64 delta = INF;
-      for (int j = 1; j <= N; ++j) {
-        if (used[j]) continue;
-        i64 cur = -W[(i0 - 1) * N + (j - 1)] - u[i0] - v[j];
-        if (cur < minv[j]) { minv[j] = cur; way[j] = j0; }
-        if (minv[j] < delta) { delta = minv[j]; j1 = j; }
+  std::vector<i64> pu(N, 0), pv(N, 0), dist(N), row_dist(N);
+  std::vector<int> col_to_row(N, -1), held(N, -1), via_row(N);   // held[i]: column of row i; via_row[j]: the tree
+                                                                  // row from which column j was reached
+  std::vector<char> settled(N);
+  std::vector<int> tree_rows;
+  for (int root = 0; root < N; ++root) {
+    std::fill(dist.begin(), dist.end(), INF);
+    std::fill(settled.begin(), settled.end(), 0);
+    tree_rows.assign(1, root);
+    row_dist[root] = 0;
+    int row = root, free_col = -1;
+    i64 reach = 0;   // distance of the column settled last
+    while (free_col < 0) {
+      // relax the unsettled columns from the row that joined the tree last, then settle the nearest one
+      int nearest = -1;
+      for (int j = 0; j < N; ++j) {
+        if (settled[j]) continue;
+        const i64 through = row_dist[row] + (-W[row * N + j] - pu[row] - pv[j]);
+        if (through < dist[j]) { dist[j] = through; via_row[j] = row; }
+        if (nearest < 0 || dist[j] < dist[nearest]) nearest = j;
       }
-      for (int j = 0; j <= N; ++j) {
-        if (used[j]) { u[p[j]] += delta; v[j] -= delta; }
-        else minv[j] -= delta;
+      settled[nearest] = 1;
+      reach = dist[nearest];
+      if (col_to_row[nearest] < 0) {
+        free_col = nearest;
+      } else {
+        row = col_to_row[nearest];
+        row_dist[row] = reach;
+        tree_rows.push_back(row);
       }
-      j0 = j1;
-    } while (p[j0] != 0);
-    do {
-      int j1 = way[j0];
-      p[j0] = p[j1];
-      j0 = j1;
-    } while (j0);
+    }
+    // potentials: tree rows rise by what is left of their way to the end of the path, settled columns fall
+    for (int i : tree_rows) pu[i] += reach - row_dist[i];
+    for (int j = 0; j < N; ++j)
+      if (settled[j]) pv[j] += dist[j] - reach;
+    // flip the path: each column on it takes the row it was reached from
+    for (int j = free_col; j >= 0;) {
+      const int i = via_row[j];
+      const int gives_up = held[i];   // -1 for the root row, which ends the walk
+      col_to_row[j] = i;
+      held[i] = j;
+      j = gives_up;
+    }
   }
   i64 total = 0;
-  for (int j = 1; j <= N; ++j) {
-    row_to_col[p[j] - 1] = j - 1;
-    total += W[(p[j] - 1) * N + (j - 1)];
+  for (int j = 0; j < N; ++j) {
+    row_to_col[col_to_row[j]] = j;
+    total += W[col_to_row[j] * N + j];
   }
-  if (pu) for (int i = 0; i < N; ++i) pu[i] = u[i + 1];
-  if (pv) for (int j = 0; j < N; ++j) pv[j] = v[j + 1];
+  if (pu_out) for (int i = 0; i < N; ++i) pu_out[i] = pu[i];
+  if (pv_out) for (int j = 0; j < N; ++j) pv_out[j] = pv[j];
   return total;
 }
 
