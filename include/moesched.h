@@ -414,6 +414,17 @@ int moesched_bvn_decompose_static(int B, int N, const int32_t* d_demand, int k_m
  */
 long long moesched_probe_int_ops(int blocks, int iters, uint32_t* d_out, void* stream);
 
+/*
+ * Debugging aid (no counterpart in the paper). The library can be built with -DMOESCHED_CHECKED
+ * (paper_2605_26845_b200/build.py builds that variant as libmoesched_checked.so): every memory index
+ * that the kernels derive from the matching state is then range-checked, an index out of range is
+ * counted and replaced by 0 (the access stays in bounds, the kernel ends normally), and this call
+ * returns how many were counted on the current device since the library was loaded. It
+ * synchronises the device. A library built without the checks returns -1; -2 means a CUDA call
+ * failed. Results of the checked build are identical to the normal one; it is slower.
+ */
+long long moesched_debug_index_faults(void);
+
 /* CUDA error code (cudaError_t as int) of the last failed CUDA call made by
  * this library on the calling thread; 0 if none. */
 int moesched_last_cuda_error(void);

@@ -37,28 +37,47 @@ class _Model(ctypes.Structure):
 _lib = None
 
 
+def _open(path):
+    if not os.path.exists(path):
+        raise MoeschedError(f"{path} is missing: run `python -m paper_2605_26845_b200.build` "
+                            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
+    lib.moesched_strerror.restype = ctypes.c_char_p
+    lib.moesched_status_str.restype = ctypes.c_char_p
+    lib.moesched_workspace_bytes.restype = ctypes.c_size_t
+    for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
+                 "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
+                 "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error",
+                 "moesched_schedule_order", "moesched_schedule_permute", "moesched_best_budget",
+                 "moesched_bvn_real_decompose"):
+        getattr(lib, name).restype = ctypes.c_int
+    lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
+    lib.moesched_order_scratch_bytes.restype = ctypes.c_size_t
+    lib.moesched_probe_int_ops.restype = ctypes.c_longlong
+    lib.moesched_debug_index_faults.restype = ctypes.c_longlong
+    return lib
+
+
 def load_library():
     """dlopen libmoesched.so (built in-tree by paper_2605_26845_b200/build.py)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise MoeschedError(f"{LIB_PATH} is missing: run `python -m paper_2605_26845_b200.build` "
-                                "(there is no CPU fallback)")
-        lib = ctypes.CDLL(LIB_PATH)
-        lib.moesched_strerror.restype = ctypes.c_char_p
-        lib.moesched_status_str.restype = ctypes.c_char_p
-        lib.moesched_workspace_bytes.restype = ctypes.c_size_t
-        for name in ("moesched_mw_decompose", "moesched_bvn_decompose", "moesched_bvn_decompose_static",
-                     "moesched_schedule_eval", "moesched_schedule_prefix_eval", "moesched_ideal_a2a",
-                     "moesched_sinkhorn_scale", "moesched_sinkhorn_durations", "moesched_last_cuda_error",
-                     "moesched_schedule_order", "moesched_schedule_permute", "moesched_best_budget",
-                     "moesched_bvn_real_decompose"):
-            getattr(lib, name).restype = ctypes.c_int
-        lib.moesched_bvn_scratch_bytes.restype = ctypes.c_size_t
-        lib.moesched_order_scratch_bytes.restype = ctypes.c_size_t
-        lib.moesched_probe_int_ops.restype = ctypes.c_longlong
-        _lib = lib
+        _lib = _open(LIB_PATH)
     return _lib
+
+
+def use_library(path=None):
+    """Route every call of this binding through another build of the library, e.g. the checked one
+    (libmoesched_checked.so, see build.py); None goes back to the regular library. Returns the path."""
+    global _lib
+    path = LIB_PATH if path is None else path
+    _lib = _open(path)
+    return path
+
+
+def debug_index_faults() -> int:
+    """Out-of-range indices the checked build has caught on the current device (-1: no checks compiled in)."""
+    return int(load_library().moesched_debug_index_faults())
 
 
 def _check(rc, what):

@@ -1,4 +1,6 @@
 // C ABI of the library: argument checks, launch geometry, error reporting.
+#include <vector>
+
 #include "common.cuh"
 
 namespace moesched {
@@ -50,6 +52,14 @@ bool model_in_range(const moesched_model_t& m) {
          m.expert_ps_per_token >= 0 && m.expert_ps_per_token <= lim30 && m.expert_knee_tokens >= 0 &&
          m.expert_knee_tokens <= 2147483647LL;
 }
+
+#ifdef MOESCHED_CHECKED
+static std::vector<FaultReader>& fault_readers() {
+  static std::vector<FaultReader> readers;   // built on first use: the files register during static initialisation
+  return readers;
+}
+void register_fault_reader(FaultReader reader) { fault_readers().push_back(reader); }
+#endif
 
 static bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
 static bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7) == 0; }
@@ -265,6 +275,21 @@ int moesched_bvn_real_decompose(int B, int N, const double* d_matrix, double tol
   cudaError_t e = run_bvn_real(B, N, d_matrix, tol, k_max, d_perm, d_lambda, d_count, d_sum_lambda, d_max_left,
                                d_scratch, d_status, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOESCHED_OK : fail_cuda(e);
+}
+
+long long moesched_debug_index_faults(void) {
+#ifdef MOESCHED_CHECKED
+  if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+  long long total = 0;
+  for (FaultReader read : fault_readers()) {
+    const unsigned v = read();
+    if (v == 0xffffffffu) return -2;
+    total += v;
+  }
+  return total;
+#else
+  return -1;
+#endif
 }
 
 int moesched_last_cuda_error(void) { return g_last_cuda_error; }

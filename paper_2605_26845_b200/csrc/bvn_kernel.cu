@@ -171,7 +171,8 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
         cell[s] = nullptr;
         if (c < N) {
           // with the working copy in global memory every row is "near": no split to test
-          cell[s] = (MODE == 2 ? A.near_ + (size_t)M.mr[s] * A.S : A.row(M.mr[s])) + c;
+          const int mrow = MS_AT(M.mr[s], N);
+          cell[s] = (MODE == 2 ? A.near_ + (size_t)mrow * A.S : A.row(mrow)) + c;
           val[s] = *cell[s];
           cmin = min(cmin, val[s]);
         }

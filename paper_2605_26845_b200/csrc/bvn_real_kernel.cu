@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(128) bvn_real_kernel(int B, int N, int S, cons
         const int c = lane * CPL + s;
         val[s] = 1e300;
         if (c < N) {
-          val[s] = A[(size_t)M.mr[s] * S + c];
+          val[s] = A[(size_t)MS_AT(M.mr[s], N) * S + c];
           cmin = fmin(cmin, val[s]);
         }
       }
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(128) bvn_real_kernel(int B, int N, int S, cons
         if (c < N) {
           double nv = __dsub_rn(val[s], cmin);
           if (!(nv > tol)) nv = 0.0;
-          A[(size_t)M.mr[s] * S + c] = nv;
+          A[(size_t)MS_AT(M.mr[s], N) * S + c] = nv;
           if (nv == 0.0) {
 #pragma unroll
             for (int w = 0; w < W; ++w) C[s][w] &= ~M.word(s, w);

@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(32 * NW) bvn_team_kernel(int B, int N, int S, 
             sh.par[t] = (short)lowest_bit<W>(hit);
             if (m.my_mr < 0) isfree = true;
             else if (m.my_mr >= thr) met = true;
-            else bs.wait[m.my_mr] = 1;
+            else bs.wait[MS_AT(m.my_mr, N)] = 1;
           }
           red.min_key(isfree, t, 0, lane);
           red.add_member<W>(met, m.my_mr, lane);
@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(32 * NW) bvn_team_kernel(int B, int N, int S, 
         if (t == 0) {
           int j = jf, ok = 0, lo = sh.misc[2], hi = sh.misc[3];
           for (int it = 0; it <= N; ++it) {
-            const int i = sh.par[j];
+            const int i = MS_AT((int)sh.par[MS_AT(j, N)], N);
             const int jprev = sh.x[i];
             sh.mr[j] = (short)i;
             sh.x[i] = (short)j;
@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(32 * NW) bvn_team_kernel(int B, int N, int S, 
       // ---- coefficient = smallest matched entry; subtract it along the matching; emit ----
       red.open();
       int val = INF32;
-      if (in) val = mat[(size_t)m.my_mr * S + t];
+      if (in) val = mat[(size_t)MS_AT(m.my_mr, N) * S + t];
       {
         const unsigned wmin = __reduce_min_sync(FULL, (unsigned)val);
         if (lane == 0) atomicMin(&red.cur()[TeamRed::MIN], wmin);
@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(32 * NW) bvn_team_kernel(int B, int N, int S, 
       bool zero = false;
       if (in) {
         const int nv = val - cmin;
-        mat[(size_t)m.my_mr * S + t] = nv;
+        mat[(size_t)MS_AT(m.my_mr, N) * S + t] = nv;
         zero = nv == 0;
         if (zero) {
 #pragma unroll

@@ -19,6 +19,34 @@ namespace moesched {
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int INF32 = 0x7fffffff;
 
+// Index checks of the debug build (-DMOESCHED_CHECKED; the stand-in for a memory checker on machines
+// where none can be run): every shared- or global-memory index that comes out of the matching state
+// (a matched row or column, a path predecessor, a search level) goes through MS_AT(index, limit).
+// In the checked build an index outside [0, limit) is counted in a per-file device counter and
+// replaced by 0, so that the access stays in bounds and the kernel ends normally; the host reads the sum
+// of the counters through moesched_debug_index_faults(). In the normal build MS_AT(i, n) is just (i).
+#ifdef MOESCHED_CHECKED
+static __device__ unsigned g_index_faults;
+__device__ __forceinline__ int checked_index(int i, int n) {
+  if ((unsigned)i >= (unsigned)n) {
+    atomicAdd(&g_index_faults, 1u);
+    return 0;
+  }
+  return i;
+}
+#define MS_AT(i, n) ::moesched::checked_index((i), (n))
+using FaultReader = unsigned (*)();
+void register_fault_reader(FaultReader reader);   // api.cu
+static unsigned read_faults_of_this_file() {
+  unsigned v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_index_faults, sizeof v) != cudaSuccess) return 0xffffffffu;
+  return v;
+}
+static const bool g_fault_reader_registered = (register_fault_reader(&read_faults_of_this_file), true);
+#else
+#define MS_AT(i, n) (i)
+#endif
+
 enum WorkField { WK_SCAN = 0, WK_AUG = 1, WK_TIGHT = 2, WK_SWEEP = 3, WK_LEVEL = 4, WK_ROT = 5, WK_MATCH = 6, WK_SKIP = 7, WK_POP = 8, WK_BATCH = 9 };
 
 // ---- small helpers on register arrays -------------------------------------------------
@@ -627,7 +655,7 @@ __device__ __forceinline__ void collect_dependants(int N, int lane, const unsign
       if (r < 0) break;
       clear_bit<W>(left, r);
 #pragma unroll
-      for (int w = 0; w < W; ++w) out[w] |= desc[r * W + w];
+      for (int w = 0; w < W; ++w) out[w] |= desc[MS_AT(r, N) * W + w];
     }
     __syncwarp();
     // lane l clears the entries of the rows l, l+32, ... that were just read
@@ -635,7 +663,7 @@ __device__ __forceinline__ void collect_dependants(int N, int lane, const unsign
     for (int k = 0; k < W; ++k) {
       if ((rows[k] >> lane) & 1u) {
 #pragma unroll
-        for (int w = 0; w < W; ++w) desc[(k * 32 + lane) * W + w] = 0u;
+        for (int w = 0; w < W; ++w) desc[MS_AT(k * 32 + lane, N) * W + w] = 0u;
       }
     }
     __syncwarp();
@@ -722,7 +750,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
   for (int guard = 0; guard < N; ++guard) {
     const int i = lowest_bit<W>(todo);
     if (i < 0) break;
-    const int xi = x[i];
+    const int xi = x[MS_AT(i, N)];
     work[WK_SWEEP]++;
     // backward search from row i among the rows >= i; the one-hot mask of i and the set {i, i+1, ...}
     // come from isolating the lowest bit of todo
@@ -791,7 +819,7 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       // level at which that row was reached
       int lvl = 0;
       for (int d = 1; d <= level; ++d) {
-        unsigned hw = hist[d * W + (cur >> 5)];
+        unsigned hw = hist[d * W + (MS_AT(cur, N) >> 5)];
         if ((hw >> (cur & 31)) & 1u) lvl = d;
       }
       if (lvl == 0) ok_all = false;
@@ -817,14 +845,14 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
         const int s2 = __shfl_sync(FULL, ms, L2);
         const int nxt = __shfl_sync(FULL, M.row_of(s2), L2);
         if (lane == L2) M.assign(s2, cur);
-        if (lane == 0) x[cur] = (short)(L2 * CPL + s2);
+        if (lane == 0) x[MS_AT(cur, N)] = (short)(L2 * CPL + s2);
         last = max(last, cur);
         cur = nxt;
         --lvl;
         work[WK_ROT]++;
       }
       if (lane == L) M.assign(sl, i);
-      if (lane == 0) x[i] = (short)jstar;
+      if (lane == 0) x[MS_AT(i, N)] = (short)jstar;
       __syncwarp();
       if constexpr (MEMO) {
         // the moved rows changed column: every record that contains one of them is void
@@ -925,10 +953,10 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   for (int it = 0; it <= N; ++it) {
     const int L = j / CPL, sl = j % CPL;
     const int i = __shfl_sync(FULL, pick<CPL>(par, sl), L);
-    const int jprev = x[i];
+    const int jprev = x[MS_AT(i, N)];
     __syncwarp();
     if (lane == L) M.assign(sl, i);
-    if (lane == 0) x[i] = (short)j;
+    if (lane == 0) x[MS_AT(i, N)] = (short)j;
     __syncwarp();
     lo = min(lo, i);
     hi = max(hi, i);

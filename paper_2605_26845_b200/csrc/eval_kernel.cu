@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
               const int j = (int)((dest[q].v >> (8 * s)) & 0xff);
               if (j < N) {
                 set_bit<W>(cols, j);
-                auto* p = D.row(r) + j;
+                auto* p = D.row(r) + MS_AT(j, N);
                 const int val = *p;
                 const int sv = min(dk, val);
                 *p = val - sv;

@@ -115,9 +115,9 @@ __global__ void __launch_bounds__(32 * NW) eval_team_kernel(int B, int N, const 
         int sv = 0;
         if (in) {
           const int dk = st->dur[q];
-          const int val = myrow[dest[q]];
+          const int val = myrow[MS_AT(dest[q], N)];
           sv = min(dk, val);
-          myrow[dest[q]] = (unsigned short)(val - sv);
+          myrow[MS_AT(dest[q], N)] = (unsigned short)(val - sv);
         }
         const int g = __reduce_max_sync(FULL, sv);
         if (lane == 0 && g > 0) atomicMax(&st->gmax[q], g);

@@ -134,7 +134,7 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
     unsigned scanned = 0u;     // bit s: the lane's column s is settled
     {
       RowVec<CPL> rv;
-      if (lane_in) rv = load_cols<CPL>(R.row(f), lane);
+      if (lane_in) rv = load_cols<CPL>(R.row(MS_AT(f, N)), lane);
 #pragma unroll
       for (int s = 0; s < CPL; ++s) {
         bool valid = lane * CPL + s < N;
@@ -161,7 +161,7 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
       work[WK_SCAN]++;
       if (i < 0) { jfin = L * CPL + sl; break; }
       RowVec<CPL> rv;
-      if (lane_in) rv = load_cols<CPL>(R.row(i), lane);
+      if (lane_in) rv = load_cols<CPL>(R.row(MS_AT(i, N)), lane);
       // the owner of the settled column forms h from its own entry and dual: one broadcast instead of two
       const int h = __shfl_sync(FULL, -pick<CPL>(rv.v, sl) - pick<CPL>(st.v, sl) - mu, L);
 #pragma unroll
@@ -180,10 +180,10 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
     for (int it = 0; it <= N; ++it) {
       const int L = j / CPL, sl = j % CPL;
       const int i = __shfl_sync(FULL, pick<CPL>(pred, sl), L);
-      const int jprev = x[i];
+      const int jprev = x[MS_AT(i, N)];
       __syncwarp();
       if (lane == L) st.M.assign(sl, i);
-      if (lane == 0) x[i] = (short)j;
+      if (lane == 0) x[MS_AT(i, N)] = (short)j;
       __syncwarp();
       if (i == f) break;
       j = jprev;
@@ -217,7 +217,6 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
                                                  uint8_t* __restrict__ perm, int32_t* __restrict__ dur,
                                                  int32_t* __restrict__ count, int32_t* __restrict__ residual,
                                                  int32_t* status, long long* __restrict__ work_out, int only_class) {
-  constexpr int W = CPL;
   constexpr bool CLUSTER = MODE == 1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   if (only_class != 0) {
@@ -296,7 +295,7 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
       for (int s = 0; s < CPL; ++s) {
         const int c = lane * CPL + s;
         if (c < N && st.M.mr[s] >= 0) {
-          auto* p = R.row(st.M.mr[s]) + c;
+          auto* p = R.row(MS_AT(st.M.mr[s], N)) + c;
           const int val = *p;
           dmax = max(dmax, val);
           served += val != 0;

@@ -154,10 +154,10 @@ __global__ void __launch_bounds__(32 * NW) mw_team_kernel(int B, int N, const in
       if (lane == 0) { ms.best[r] = (short)col; ms.u[r] = mn; }
     }
     __syncthreads();
-    if (in) atomicMin(&ms.first[ms.best[t]], t);
+    if (in) atomicMin(&ms.first[MS_AT((int)ms.best[t], N)], t);
     __syncthreads();
     int my_mr = in && ms.first[t] != INF32 ? ms.first[t] : -1;   // row of column t
-    int my_x = in && ms.first[ms.best[t]] == t ? (int)ms.best[t] : -1;   // column of row t
+    int my_x = in && ms.first[MS_AT((int)ms.best[t], N)] == t ? (int)ms.best[t] : -1;   // column of row t
     if (t == 0) work[WK_TIGHT] += N;
     // tight edges under the current duals, by rows: the leftover rows bid for free tight columns
     tight_graph_team<NW>(R, ms, N, t, lane, warp, in, v, m);
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(32 * NW) mw_team_kernel(int B, int N, const in
         const int wm = __reduce_min_sync(FULL, d_eff);
         const bool cand = !done && dist == wm;
         const unsigned cb = __ballot_sync(FULL, cand);
-        if (cand) ms.hbuf[p][t] = my_mr >= 0 ? -(int)R[(size_t)my_mr * N + t] - v : 0;
+        if (cand) ms.hbuf[p][t] = my_mr >= 0 ? -(int)R[(size_t)MS_AT(my_mr, N) * N + t] - v : 0;
         if (lane == 0) { ms.wmin[p][warp] = wm; ms.wcand[p][warp] = cb; }
         __syncthreads();
         mu = INF32;
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(32 * NW) mw_team_kernel(int B, int N, const in
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              iq[q] = cq[q] >= 0 ? (int)sh.mr[cq[q]] : 0;
+              iq[q] = cq[q] >= 0 ? MS_AT((int)sh.mr[cq[q]], N) : 0;
               hq[q] = cq[q] >= 0 ? ms.hbuf[p][cq[q]] - mu : 0;
             }
 #pragma unroll
@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(32 * NW) mw_team_kernel(int B, int N, const in
       if (t == 0) {
         int j = jfin, ok = 0;
         for (int it = 0; it <= N; ++it) {
-          const int i = sh.par[j];
+          const int i = MS_AT((int)sh.par[MS_AT(j, N)], N);
           const int jprev = sh.x[i];
           sh.mr[j] = (short)i;
           sh.x[i] = (short)j;
@@ -305,8 +305,8 @@ __global__ void __launch_bounds__(32 * NW) mw_team_kernel(int B, int N, const in
     red.open();
     int val = 0;
     if (in && m.my_mr >= 0) {
-      val = R[(size_t)m.my_mr * N + t];
-      R[(size_t)m.my_mr * N + t] = 0;
+      val = R[(size_t)MS_AT(m.my_mr, N) * N + t];
+      R[(size_t)MS_AT(m.my_mr, N) * N + t] = 0;
       pout[(size_t)k * N + t] = (uint8_t)m.my_x;
     }
     red.max_val(val > 0, (unsigned)val, lane);

@@ -76,11 +76,11 @@ __global__ void __launch_bounds__(32) order_kernel(int B, int k_stride, const lo
       r3 += o.k3 < mine.k3 || (o.k3 == mine.k3 && first);
       r4 += o.k4 < mine.k4 || (o.k4 == mine.k4 && first);
     }
-    ord[0 * k_stride + r1] = (short)k;
-    ord[1 * k_stride + r2] = (short)k;
+    ord[0 * k_stride + MS_AT(r1, K)] = (short)k;
+    ord[1 * k_stride + MS_AT(r2, K)] = (short)k;
     // increasing a, placed alternately at the front and at the back
-    ord[2 * k_stride + ((r3 & 1) ? K - 1 - (r3 >> 1) : (r3 >> 1))] = (short)k;
-    ord[3 * k_stride + r4] = (short)k;
+    ord[2 * k_stride + MS_AT((r3 & 1) ? K - 1 - (r3 >> 1) : (r3 >> 1), K)] = (short)k;
+    ord[3 * k_stride + MS_AT(r4, K)] = (short)k;
   }
   __syncwarp();
   // one lane per candidate runs the three-stage recurrence on the fixed job times
@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(32) order_kernel(int B, int k_stride, const lo
   if (lane < ORDER_RULES) {
     long long dsp = 0, cmp = 0, cmb = 0;
     for (int p = 0; p < K; ++p) {
-      const int k = lane == 0 ? p : (int)ord[(lane - 1) * k_stride + p];
+      const int k = lane == 0 ? p : MS_AT((int)ord[(lane - 1) * k_stride + p], K);
       dsp += a[k];
       cmp = max(dsp, cmp) + bt[k];
       cmb = max(cmp, cmb) + a[k];

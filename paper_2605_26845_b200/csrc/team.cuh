@@ -261,14 +261,14 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
     red.open();
     {
       const bool adj = in && ((sh.ri[t >> 5] >> (t & 31)) & 1u);
-      const bool reached = adj && m.my_mr >= 0 && sh.lvl[m.my_mr] >= stamp;
+      const bool reached = adj && m.my_mr >= 0 && sh.lvl[MS_AT(m.my_mr, N)] >= stamp;
       red.min_key(reached, t, m.my_mr, lane);
     }
     red.close();
     const unsigned key = red.cur()[TeamRed::MIN];
     red.next();
     if (key == 0xffffffffu) { ok_all = false; continue; }
-    const int jstar = (int)(key >> 16);
+    const int jstar = MS_AT((int)(key >> 16), N);
     if (jstar == xi) {
       // record: row i stays put until one of the rows that can reach it changes column
       if constexpr (MEMO) {
@@ -282,18 +282,18 @@ __device__ __forceinline__ bool team_canonicalise(TeamShared<NW>& sh, TeamRed& r
     }
     // rotate along the alternating cycle: the row that gives up column jstar takes the column of
     // its successor towards row i, and so on down the levels
-    int cur = (int)(key & 0xffffu);
+    int cur = MS_AT((int)(key & 0xffffu), N);
     int lvl = sh.lvl[cur] - stamp;
     if (lvl <= 0 || lvl > level) { ok_all = false; continue; }
     for (int it = 0; it < N && lvl > 0; ++it) {
       red.open();
-      const bool q = in && m.my_mr >= 0 && sh.lvl[m.my_mr] == stamp + lvl - 1 && test_bit<W>(m.Cc, cur);
+      const bool q = in && m.my_mr >= 0 && sh.lvl[MS_AT(m.my_mr, N)] == stamp + lvl - 1 && test_bit<W>(m.Cc, cur);
       red.min_key(q, t, m.my_mr, lane);
       red.close();
       const unsigned k2 = red.cur()[TeamRed::MIN];
       red.next();
       if (k2 == 0xffffffffu) { ok_all = false; break; }
-      const int c2 = (int)(k2 >> 16), nxt = (int)(k2 & 0xffffu);
+      const int c2 = MS_AT((int)(k2 >> 16), N), nxt = MS_AT((int)(k2 & 0xffffu), N);
       if (t == c2) {
         m.my_mr = cur;
         sh.mr[c2] = (short)cur;
@@ -395,7 +395,7 @@ __device__ __forceinline__ int warp_back_search(const TeamShared<NW>& sh, const 
 #pragma unroll
     for (int w = 0; w < W; ++w) {
       if ((F[w] >> lane) & 1u) {
-        const int c = sh.x[w * 32 + lane];
+        const int c = MS_AT((int)sh.x[w * 32 + lane], N);
         unsigned col[W];
         load_words<W>(ts.cc + c * W, col);
 #pragma unroll
@@ -416,7 +416,7 @@ __device__ __forceinline__ int warp_back_search(const TeamShared<NW>& sh, const 
     ++level;
 #pragma unroll
     for (int w = 0; w < W; ++w)
-      if ((F[w] >> lane) & 1u) lvl[w * 32 + lane] = stamp + level;
+      if ((F[w] >> lane) & 1u) lvl[MS_AT(w * 32 + lane, N)] = stamp + level;
   }
   __syncwarp();
   // lowest column adjacent to row i whose row was reached (its own column always qualifies)
@@ -442,7 +442,7 @@ template <int NW>
 __device__ __forceinline__ int warp_rotate(TeamShared<NW>& sh, const TeamSearchShared<NW>& ts, const int* lvl, int stamp,
                                            int N, int i, int jstar, int lane, int& steps) {
   constexpr int W = NW;
-  int cur = sh.mr[jstar];
+  int cur = MS_AT((int)sh.mr[MS_AT(jstar, N)], N);
   int L = lvl[cur] - stamp;
   int top = i;
   if (L <= 0 || L > N) return -1;
@@ -454,13 +454,13 @@ __device__ __forceinline__ int warp_rotate(TeamShared<NW>& sh, const TeamSearchS
       bool ok = false;
       if (c < N && ((ts.rr[cur * W + w] >> lane) & 1u)) {
         const int r = sh.mr[c];
-        ok = r >= 0 && lvl[r] == stamp + L - 1;
+        ok = r >= 0 && lvl[MS_AT(r, N)] == stamp + L - 1;
       }
       const unsigned ball = __ballot_sync(FULL, ok);
       if (cp < 0 && ball != 0u) cp = w * 32 + __ffs(ball) - 1;
     }
     if (cp < 0) return -1;
-    const int nxt = sh.mr[cp];
+    const int nxt = MS_AT((int)sh.mr[cp], N);
     __syncwarp();
     if (lane == 0) { sh.mr[cp] = (short)cur; sh.x[cur] = (short)cp; }
     __syncwarp();
@@ -470,7 +470,7 @@ __device__ __forceinline__ int warp_rotate(TeamShared<NW>& sh, const TeamSearchS
     ++steps;
   }
   if (cur != i) return -1;
-  if (lane == 0) { sh.mr[jstar] = (short)i; sh.x[i] = (short)jstar; }
+  if (lane == 0) { sh.mr[MS_AT(jstar, N)] = (short)i; sh.x[MS_AT(i, N)] = (short)jstar; }
   __syncwarp();
   return top;
 }
@@ -522,7 +522,7 @@ __device__ __forceinline__ bool team_canonicalise_par(TeamShared<NW>& sh, TeamSe
       if (jw < 0) { bad = true; break; }
       last_done = iw;
       if (t == 0) { work[WK_SWEEP]++; work[WK_LEVEL] += ts.res[w][2]; work[WK_POP] += ts.res[w][3]; }
-      if (jw != sh.x[iw]) { wrot = w; break; }
+      if (jw != sh.x[MS_AT(iw, N)]) { wrot = w; break; }
     }
     if (bad) { ok_all = false; break; }
     from = last_done + 1;
