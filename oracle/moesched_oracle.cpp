@@ -592,7 +592,7 @@ void order_one(int N, const int32_t* D, int K, const uint8_t* perm, const int32_
 
 // ---------------------------------------------------------------------------
 // Birkhoff-von Neumann decomposition of a real-valued matrix [Sec. 3.1: A = sum_k lambda_k P_k for a
-// doubly stochastic A; Sec. 4.2 speaks of its coefficients, "around 0.03" on an 8 x 8 matrix]. The
+// doubly stochastic A; Sec. 4.2 reports coefficients of a few hundredths on an 8 x 8 matrix]. The
 // input is what Sinkhorn-Knopp scaling returns, doubly stochastic only up to the error of its last
 // sweep, so two things the integer version does not need are stated here: entries at or below `tol`
 // count as zero (on input, and after each subtraction), and the loop also ends when the support has

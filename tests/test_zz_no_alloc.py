@@ -48,7 +48,7 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row():
 
 
 def test_static_entry_point_against_the_oracle_without_touching_device_memory():
-    """The CPU oracle is the judge here, not the sibling entry point; and the call must leave the
+    """Checked against the CPU oracle here, not against the sibling entry point; and the call must leave the
     amount of free device memory exactly as it found it, which is the whole point for a caller
     that cannot allocate. Two shapes: small matrices (one warp per matrix, four matrices per
     CTA) and 200 ranks in a batch of two (one CTA of eight warps per matrix)."""
