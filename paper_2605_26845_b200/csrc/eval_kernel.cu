@@ -84,9 +84,9 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
   int lane, b;
   bool loaded = true;
   if constexpr (MODE == 2) {
-    WarpCtx16 cx = warp_prologue16<CPL>(B, N, S, demand, smem_raw);
+    WarpCtx16 cx = warp_prologue16<CPL, true>(B, N, S, demand, smem_raw);
     if (!cx.worker) return;
-    lane = cx.lane; b = cx.b; D = cx.M;
+    lane = cx.lane; b = cx.b; D = cx.M; loaded = cx.loaded;
   } else {
     WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
     if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }

@@ -230,9 +230,9 @@ __global__ void __launch_bounds__(128) mw_kernel(int B, int N, int S, const int3
   unsigned* hist;
   bool loaded = true;
   if constexpr (MODE == 2) {
-    WarpCtx16 cx = warp_prologue16<CPL>(B, N, S, demand, smem_raw);
+    WarpCtx16 cx = warp_prologue16<CPL, false>(B, N, S, demand, smem_raw);
     if (!cx.worker) return;
-    lane = cx.lane; b = cx.b; R = cx.M; x = cx.x; hist = cx.hist;
+    lane = cx.lane; b = cx.b; R = cx.M; x = cx.x; hist = cx.hist; loaded = cx.loaded;
   } else {
     WarpCtx cx = warp_prologue<CPL, CLUSTER>(B, N, S, demand, smem_raw);
     if (!cx.worker) { cluster_epilogue<CLUSTER>(); return; }
