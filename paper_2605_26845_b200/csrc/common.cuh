@@ -1059,6 +1059,123 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   return false;
 }
 
+// ---- repair of a matching that lost ONE edge, canonical for the row that lost it ------------------------
+// Birkhoff step: the entry (r0, c0) of a lexicographically smallest perfect matching has just vanished, so
+// row r0 and column c0 are free and every other row is matched. Rows below r0 keep their columns (they did so
+// with more edges available). The columns that CAN be handed to r0 without touching rows below it are found
+// by one forward search from the free column over the rows above r0: a row adjacent to a column of the
+// previous level could move there and release its own column. r0 takes the lowest such column it is adjacent
+// to -- which is its column in the lexicographically smallest matching of the new graph -- and the rows on the
+// way each move one step towards c0. This replaces an arbitrary augmenting path followed by a search (and
+// usually a rotation) for row r0. Returns 1 when done (hi = highest row moved, `changed` gets the moved rows),
+// 0 when r0 cannot be re-matched without rows below it (the caller falls back to augment_from), -1 if an
+// iteration limit was hit.
+template <int CPL>
+__device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const unsigned (&C)[CPL][CPL], Match<CPL>& M,
+                                                short* x, unsigned* hist, int& hi, unsigned (&changed)[CPL],
+                                                unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+  constexpr int W = CPL;
+  unsigned alive[W], r0mask[W];
+  ge_mask<W>(r0 + 1, alive);        // rows above r0 not reached yet
+  onehot_mask<W>(r0, r0mask);
+  unsigned front = 0u;              // bit s: the lane's column s belongs to the current level
+#pragma unroll
+  for (int s = 0; s < CPL; ++s)
+    if (lane * CPL + s < N && M.mr[s] < 0) front |= 1u << s;
+  if (__popc(__ballot_sync(FULL, front != 0u)) != 1 || __popc(front) > 1) return 0;   // exactly one free column
+  unsigned freeable = front;        // bit s: column s is free or can be released
+  int level = 0;
+  for (int it = 0; it < N; ++it) {
+    unsigned acc[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+    for (int s = 0; s < CPL; ++s) {
+      if ((front >> s) & 1u) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
+      }
+    }
+    unsigned nw[W];
+    bool grew = false;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      nw[w] = __reduce_or_sync(FULL, acc[w]) & alive[w];
+      alive[w] &= ~nw[w];
+      grew |= nw[w] != 0u;
+    }
+    work[WK_SCAN]++;
+    if (!grew) break;
+    ++level;
+    hist_store<W>(hist, level, nw, lane);
+    front = 0u;
+#pragma unroll
+    for (int s = 0; s < CPL; ++s)
+      if (M.mr[s] >= 0 && M.in(nw, s)) front |= 1u << s;
+    freeable |= front;
+  }
+  __syncwarp();
+  // the lowest column that r0 is adjacent to and that can be released
+  int myslot = -1;
+#pragma unroll
+  for (int ss = 0; ss < CPL; ++ss) {
+    const int s = CPL - 1 - ss;
+    if (((freeable >> s) & 1u) && intersects<W>(C[s], r0mask)) myslot = s;
+  }
+  const unsigned ball = __ballot_sync(FULL, myslot >= 0);
+  if (ball == 0u) return 0;
+  const int L = __ffs(ball) - 1;
+  const int sl = __shfl_sync(FULL, myslot, L);
+  int cur = __shfl_sync(FULL, M.row_of(sl), L);   // the row that gives that column up
+  if (lane == L) M.assign(sl, r0);
+  if (lane == 0) x[MS_AT(r0, N)] = (short)(L * CPL + sl);
+  set_bit<W>(changed, r0);
+  hi = max(hi, r0);
+  if (cur < 0) return 1;   // r0 took the free column itself
+  int lvl = 0;
+  for (int d = 1; d <= level; ++d) {
+    const unsigned hw = hist[d * W + (MS_AT(cur, N) >> 5)];
+    if ((hw >> (cur & 31)) & 1u) lvl = d;
+  }
+  if (lvl == 0) return -1;
+  for (int it = 0; it <= N; ++it) {
+    // cur, reached at level lvl, moves to a column of level lvl - 1 (level 0: the free column)
+    unsigned cmask[W];
+    onehot_mask<W>(cur, cmask);
+    int ms = -1;
+    if (lvl == 1) {
+#pragma unroll
+      for (int ss = 0; ss < CPL; ++ss) {
+        const int s = CPL - 1 - ss;
+        if (lane * CPL + s < N && M.mr[s] < 0 && intersects<W>(C[s], cmask)) ms = s;
+      }
+    } else {
+      unsigned Hm[W];
+      hist_load<W>(hist, lvl - 1, Hm);
+#pragma unroll
+      for (int ss = 0; ss < CPL; ++ss) {
+        const int s = CPL - 1 - ss;
+        if (M.in(Hm, s) && intersects<W>(C[s], cmask)) ms = s;
+      }
+    }
+    const unsigned b2 = __ballot_sync(FULL, ms >= 0);
+    if (b2 == 0u) return -1;
+    const int L2 = __ffs(b2) - 1;
+    const int s2 = __shfl_sync(FULL, ms, L2);
+    const int nxt = __shfl_sync(FULL, M.row_of(s2), L2);
+    if (lane == L2) M.assign(s2, cur);
+    if (lane == 0) x[MS_AT(cur, N)] = (short)(L2 * CPL + s2);
+    set_bit<W>(changed, cur);
+    hi = max(hi, cur);
+    work[WK_AUG]++;
+    if (lvl == 1) { __syncwarp(); return 1; }
+    if (nxt < 0) return -1;
+    cur = nxt;
+    --lvl;
+  }
+  return -1;
+}
+
 // Time of one expert batch of g tokens (see moesched_model_t).
 __device__ __forceinline__ long long batch_time_ns(const moesched_model_t& m, long long g) {
   if (g <= 0) return 0;
