@@ -110,6 +110,18 @@ __global__ void __launch_bounds__(128) bvn_real_kernel(int B, int N, int S, cons
     bool exhausted = false;   // the support has no perfect matching any more
     while (nnz > 0 && k < k_max) {
       bool okm = true;
+      int nfree = 0;
+#pragma unroll
+      for (int w = 0; w < W; ++w) nfree += __popc(freerows[w]);
+      if (nfree == 1 && k > 0) {   // a single row lost its entry: re-match it canonically at once
+        const int r0 = lowest_bit<W>(freerows);
+        const int rc = canonical_repair<CPL>(N, lane, r0, C, M, x, hist, hi_changed, memo.changed, work);
+        if (rc < 0) { st_code = MOESCHED_ST_INTERNAL; break; }
+        if (rc == 1) {
+          clear_bit<W>(freerows, r0);
+          lo_changed = r0 + 1;
+        }
+      }
       for (int it = 0; it < N; ++it) {
         const int f = lowest_bit<W>(freerows);
         if (f < 0) break;
