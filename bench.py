@@ -162,8 +162,8 @@ def scalar_model_ops(work_mw, work_bvn, N):
 
 WORK_NAMES_MW = ("column_scans", "augmentations", "rows_bid", "searches", "search_levels", "rotation_steps",
                  "matchings", "rows_matched_on_tight_edges", "frontier_pops", "settled_groups")
-WORK_NAMES_BVN = ("repair_levels", "repair_path_steps", "unused", "searches", "search_levels", "rotation_steps",
-                  "matchings", "rows_skipped_as_prefix", "frontier_pops", "unused")
+WORK_NAMES_BVN = ("repair_levels", "repair_path_steps", "canonical_repairs", "searches", "search_levels",
+                  "rotation_steps", "matchings", "rows_skipped_as_prefix", "frontier_pops", "repair_fallbacks")
 
 
 def per_matching(work, names):

@@ -151,12 +151,13 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
  *                   are undefined afterwards; calls that overlap in time need
  *                   separate scratch.
  *   d_status   out  [B] int32
- *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64, may be NULL: 0 augmenting
- *                   search levels, 1 augmenting-path steps, 2 matchings
- *                   repaired, 3 canonicalisation sweeps that searched,
+ *   d_work     out  [B][MOESCHED_WORK_FIELDS] int64, may be NULL: 0 levels of the
+ *                   repair searches, 1 rows moved by the repairs, 2 rows re-matched
+ *                   canonically at once, 3 canonicalisation sweeps that searched,
  *                   4 search levels, 5 rotation steps, 6 matchings, 7 rows
  *                   skipped as unchanged prefix, 8 rows expanded by the
- *                   canonicalisation searches (frontier pops), 9 unused
+ *                   canonicalisation searches (frontier pops), 9 canonical
+ *                   re-matchings that had to fall back to the general search
  */
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                            int32_t* d_coef, int32_t* d_count, int32_t* d_aug, int32_t* d_scratch,

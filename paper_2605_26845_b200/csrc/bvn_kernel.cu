@@ -148,17 +148,19 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
     while (nnz > 0 && k < k_max) {
       // re-match the free rows: a single row that lost its entry is re-matched canonically at once
       bool okm = true;
-      int nfree = 0;
-#pragma unroll
-      for (int w = 0; w < W; ++w) nfree += __popc(freerows[w]);
-      if (nfree == 1 && k > 0) {
-        const int r0 = lowest_bit<W>(freerows);
-        const int rc = canonical_repair<CPL>(N, lane, r0, C, M, x, hist, hi_changed, memo.changed, work);
-        if (rc < 0) { st_code = MOESCHED_ST_INTERNAL; break; }
-        if (rc == 1) {
+      if (k > 0) {
+        // rows that lost their entry are re-matched canonically, lowest first, as long as that works
+        for (int it = 0; it < N; ++it) {
+          const int r0 = lowest_bit<W>(freerows);
+          if (r0 < 0) break;
+          const int rc = canonical_repair<CPL>(N, lane, r0, C, M, x, hist, hi_changed, memo.changed, work);
+          if (rc < 0) { okm = false; break; }
+          if (rc == 0) { work[WK_BATCH]++; break; }   // needs rows below r0: the general search below takes over
+          work[WK_TIGHT]++;
           clear_bit<W>(freerows, r0);
-          lo_changed = r0 + 1;   // row r0 has its final column; the rows that moved lie above it
+          lo_changed = min(lo_changed, r0 + 1);   // row r0 has its final column; the rows that moved lie above it
         }
+        if (!okm) { st_code = MOESCHED_ST_INTERNAL; break; }
       }
       for (int it = 0; it < N; ++it) {
         const int f = lowest_bit<W>(freerows);

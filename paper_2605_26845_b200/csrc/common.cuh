@@ -1059,14 +1059,17 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
   return false;
 }
 
-// ---- repair of a matching that lost ONE edge, canonical for the row that lost it ------------------------
+// ---- repair of a matching that lost an edge, canonical for the row that lost it -------------------------
 // Birkhoff step: the entry (r0, c0) of a lexicographically smallest perfect matching has just vanished, so
-// row r0 and column c0 are free and every other row is matched. Rows below r0 keep their columns (they did so
-// with more edges available). The columns that CAN be handed to r0 without touching rows below it are found
-// by one forward search from the free column over the rows above r0: a row adjacent to a column of the
-// previous level could move there and release its own column. r0 takes the lowest such column it is adjacent
-// to -- which is its column in the lexicographically smallest matching of the new graph -- and the rows on the
-// way each move one step towards c0. This replaces an arbitrary augmenting path followed by a search (and
+// row r0 and column c0 are free. Rows below r0 keep their columns (they did so with more edges available).
+// The columns that CAN be handed to r0 without touching rows below it are found by one forward search from
+// the free column(s) over the rows above r0: a row adjacent to a column of the previous level could move
+// there and release its own column. r0 takes the lowest such column it is adjacent to -- which is its column
+// in the lexicographically smallest matching of the new graph -- and the rows on the way each move one step
+// towards a free column. (When several entries vanished at once the free rows are handled lowest first; a
+// free row above r0 releases nothing and is simply passed over. Each row's choice is the lowest among the
+// matchings that leave the other free rows out, hence also among the complete ones if the rest can still be
+// matched above it; if not, the caller's general search lowers the window as far as it has to.) This replaces an arbitrary augmenting path followed by a search (and
 // usually a rotation) for row r0. Returns 1 when done (hi = highest row moved, `changed` gets the moved rows),
 // 0 when r0 cannot be re-matched without rows below it (the caller falls back to augment_from), -1 if an
 // iteration limit was hit.
@@ -1082,7 +1085,7 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
 #pragma unroll
   for (int s = 0; s < CPL; ++s)
     if (lane * CPL + s < N && M.mr[s] < 0) front |= 1u << s;
-  if (__popc(__ballot_sync(FULL, front != 0u)) != 1 || __popc(front) > 1) return 0;   // exactly one free column
+  if (__ballot_sync(FULL, front != 0u) == 0u) return 0;   // no free column: nothing to hand out
   unsigned freeable = front;        // bit s: column s is free or can be released
   int level = 0;
   for (int it = 0; it < N; ++it) {
