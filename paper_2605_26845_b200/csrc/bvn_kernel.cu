@@ -8,6 +8,8 @@
 // matching over the window of rows whose column changed (rows before the first
 // changed row provably keep theirs; rows after the last one were settled earlier
 // and removing edges cannot unsettle them).
+#include <atomic>
+
 #include "common.cuh"
 
 namespace moesched {
@@ -16,12 +18,28 @@ namespace moesched {
 // in global memory (scratch), which leaves room for many more warps per SM.
 // COUNT: the per-matrix work counters are wanted (they are plain register increments that the
 // compiler drops, registers included, when nothing reads them).
-template <int CPL, int MODE, bool COUNT>
+//
+// PACE. The warp schedulers of an SM serve their resident warps in a fixed order of preference. With several
+// equally long decompositions per scheduler the preferred warps run at full speed and finish early, and the
+// others are left to finish alone, each stalled on its own dependent chain with most issue slots empty
+// (measured, N = 64, B = 4096, all warps resident from the start: the warps in the first four slots of an SM
+// finish after 22.7 ms, those in the last four after 39.3 ms). When the whole batch is resident at once the
+// launcher therefore switches pacing on: every warp publishes, every PACE_EVERY matchings, how many entries its
+// matrix has left, reads the figures of the warps that share its scheduler (warp slot modulo 4), and sleeps for a
+// moment when it is well ahead of the slowest of them. The slots go to the warps behind and all finish together
+// (40.5 -> 38.9 ms). A sleep is a plain delay, never a wait for another warp: results and termination do not
+// depend on it. Entries carry the launch's number, so figures left by another launch are ignored.
+constexpr int PACE_EVERY = 16;          // matchings between two looks (a power of two)
+constexpr unsigned PACE_SLACK = 32;     // entries a warp may be ahead before it sleeps
+constexpr unsigned PACE_NS_PER_ENTRY = 2000, PACE_NS_MAX = 200000;
+__device__ unsigned long long g_pace[256][64];   // [SM][warp slot] = launch number << 32 | entries left
+
+template <int CPL, int MODE, bool COUNT, bool PACE = false>
 __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                   uint8_t* __restrict__ perm, int32_t* __restrict__ coef,
                                                   int32_t* __restrict__ count, int32_t* __restrict__ aug,
                                                   int32_t* scratch, int32_t* __restrict__ status,
-                                                  long long* __restrict__ work_out) {
+                                                  long long* __restrict__ work_out, unsigned pace_launch = 0u) {
   constexpr int W = CPL;
   constexpr bool CLUSTER = MODE == 1;
   constexpr bool USE_MEMO = true;
@@ -146,6 +164,25 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
     }
 
     while (nnz > 0 && k < k_max) {
+      if constexpr (PACE) {
+        if ((k & (PACE_EVERY - 1)) == 0) {
+          unsigned pace_sm, pace_slot;   // read afresh every time rather than kept in registers across the loop
+          asm volatile("mov.u32 %0, %%smid;" : "=r"(pace_sm));
+          asm volatile("mov.u32 %0, %%warpid;" : "=r"(pace_slot));
+          pace_sm &= 255u;
+          pace_slot &= 63u;
+          if (lane == 0) g_pace[pace_sm][pace_slot] = ((unsigned long long)pace_launch << 32) | (unsigned)nnz;
+          unsigned left = 0u;
+          if (lane < 16) {
+            const unsigned long long v =
+                *reinterpret_cast<const volatile unsigned long long*>(&g_pace[pace_sm][(pace_slot & 3u) + 4u * lane]);
+            if ((unsigned)(v >> 32) == pace_launch) left = (unsigned)v;
+          }
+          left = __reduce_max_sync(FULL, left);   // the most entries left among the warps of this scheduler
+          if (left > (unsigned)nnz + PACE_SLACK)
+            __nanosleep(min((left - (unsigned)nnz - PACE_SLACK) * PACE_NS_PER_ENTRY, PACE_NS_MAX));
+        }
+      }
       // re-match the free rows: a single row that lost its entry is re-matched canonically at once
       bool okm = true;
       if (k > 0) {
@@ -233,6 +270,12 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
   }
 
   if (st_code == MOESCHED_ST_BAD_INPUT) k = 0;
+  if constexpr (PACE) {   // this warp no longer counts (it may have moved on without entering the loop)
+    unsigned sm, slot;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+    asm volatile("mov.u32 %0, %%warpid;" : "=r"(slot));
+    if (lane == 0) g_pace[sm & 255u][slot & 63u] = 0ull;
+  }
   if (lane == 0) {
     count[b] = k;
     status[b] = st_code;
@@ -248,6 +291,14 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
 
 // ---- host side ---------------------------------------------------------------------------
 
+// Number of this paced launch (never 0; entries of the pacing table with another number are ignored).
+static unsigned next_pace_launch() {
+  static std::atomic<unsigned> n{0u};
+  unsigned v = ++n;
+  if (v == 0u) v = ++n;
+  return v;
+}
+
 cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* perm, int32_t* coef, int32_t* count,
                     int32_t* aug, int32_t* scratch, int32_t* status, long long* work, cudaStream_t stream) {
   Geometry ge = plan_geometry(N);
@@ -255,9 +306,9 @@ cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* per
   do {                                                                                                        \
     if (work != nullptr)                                                                                      \
       return launch_warp_kernel(bvn_kernel<C, M, true>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, \
-                                count, aug, scratch, status, work);                                           \
+                                count, aug, scratch, status, work, 0u);                                       \
     return launch_warp_kernel(bvn_kernel<C, M, false>, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef,  \
-                              count, aug, scratch, status, work);                                             \
+                              count, aug, scratch, status, work, 0u);                                         \
   } while (0)
   // Above 128 ranks a batch that leaves most SMs with a single warp goes to the kernel that puts a
   // CTA of eight warps on each matrix (measured at N = 256, B = 256: 1.0 s against 1.8 s; at N = 128,
@@ -272,6 +323,27 @@ cudaError_t run_bvn(int B, int N, const int32_t* demand, int k_max, uint8_t* per
     // a small batch is spread one matrix per CTA so that no SM sits idle
     ge.wpb = B >= 16 * sm_count() ? 4 : 1;
     ge.smem = warp_smem_bytes_global(N, ge.cpl) * ge.wpb;
+    // pacing (see PACE above) when every scheduler gets three warps or more and the whole batch is resident at once
+    if (work == nullptr && B >= 12 * sm_count()) {
+#define MOESCHED_PACED(C)                                                                                          \
+  do {                                                                                                             \
+    int per_sm = 0;                                                                                                \
+    auto kern = bvn_kernel<C, 2, false, true>;                                                                     \
+    cudaError_t eo = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ge.smem);        \
+    if (eo == cudaSuccess) eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * ge.wpb, ge.smem); \
+    if (eo != cudaSuccess) return eo;                                                                              \
+    if ((long long)per_sm * sm_count() >= (B + ge.wpb - 1) / ge.wpb)                                               \
+      return launch_warp_kernel(kern, ge, B, stream, B, N, ge.S, demand, k_max, perm, coef, count, aug, scratch,   \
+                                status, work, next_pace_launch());                                                 \
+  } while (0)
+      switch (ge.cpl) {
+        case 1: MOESCHED_PACED(1); break;
+        case 2: MOESCHED_PACED(2); break;
+        case 4: MOESCHED_PACED(4); break;
+        default: MOESCHED_PACED(8); break;
+      }
+#undef MOESCHED_PACED
+    }
     switch (ge.cpl) {
       case 1: MOESCHED_GO(1, 2);
       case 2: MOESCHED_GO(2, 2);
