@@ -108,6 +108,28 @@ def test_one_warp_kernel_above_128_ranks_in_a_large_batch(N, kw):
     assert (wide.extra[:37].cpu().numpy() == rv["aug"]).all()
 
 
+@pytest.mark.parametrize("N,per_sm", [(16, 14), (64, 13), (64, 27)])
+def test_paced_launch_of_a_resident_batch_gives_the_same_schedules(N, per_sm):
+    """From twelve matrices per SM up, when the whole batch is resident at once, the warps that share a
+    scheduler pace one another (a warp that is ahead sleeps). Timing only: the complete schedules must equal
+    those of the same matrices decomposed in a small, unpaced batch, and the oracle's."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    base = random_matrices(29, N, seed=8300 + N, **(KINDS[2] if N == 16 else KINDS[0]))
+    reps = -(-per_sm * sms // base.shape[0])
+    D = np.concatenate([base] * reps)
+    assert D.shape[0] >= 12 * sms
+    K = bvn_capacity(N)
+    rv = oracle.bvn_decompose(base, K, threads=8)
+    small = ms.bvn_decompose(dev(base), K)
+    assert_schedule_equal(small, rv, "coef")
+    for _ in range(2):   # twice: entries of the pacing table left by the first launch must not matter
+        wide = ms.bvn_decompose(dev(D), K)
+        torch.cuda.synchronize()
+        for q in range(reps):
+            part = ms.Schedule(*(getattr(wide, f)[q * 29:(q + 1) * 29] for f in ("perm", "dur", "count", "status")))
+            assert_schedule_equal(part, rv, "coef")
+
+
 @pytest.mark.parametrize("N", [233, 256])
 def test_wide_entries_above_232_ranks_run_deep_on_the_cluster_path(N):
     """Entries beyond 16 bits at N > 232 put the matrix (as int32) across the two CTAs of a cluster, for
