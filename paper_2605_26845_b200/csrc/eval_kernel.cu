@@ -18,6 +18,35 @@ __device__ __forceinline__ long long warp_sum64(long long v) {
   return v;
 }
 
+// The stage recurrences x_k = max(a_k, x_{k-1}) + b_k are compositions of maps x -> max(x + p, q) (p = b_k,
+// q = a_k + b_k), and such maps compose to a map of the same form: (p2, q2) after (p1, q1) is
+// (p1 + p2, max(q1 + p2, q2)). An inclusive scan over the lanes (five steps) therefore gives every matching of a
+// chunk its value at once, in exact integer arithmetic, instead of 32 dependent steps.
+struct MaxPlus {
+  long long p, q;
+};
+constexpr long long MAXPLUS_NONE = -(1LL << 62);   // q of the identity map (p = 0)
+__device__ __forceinline__ MaxPlus maxplus_scan(MaxPlus m, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long up_p = __shfl_up_sync(FULL, m.p, o);
+    const long long up_q = __shfl_up_sync(FULL, m.q, o);
+    if (lane >= o) {   // the maps of the lower lanes act first
+      m.q = max(up_q + m.p, m.q);
+      m.p += up_p;
+    }
+  }
+  return m;
+}
+__device__ __forceinline__ long long prefix_sum64(long long v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long up = __shfl_up_sync(FULL, v, o);
+    if (lane >= o) v += up;
+  }
+  return v;
+}
+
 template <int CPL, typename View>
 __device__ __forceinline__ long long matrix_sum(const View& M, int N, int lane, bool lane_in, int* any_negative) {
   long long acc = 0;
@@ -185,23 +214,24 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
       dur_sum += warp_sum64((long long)dk_mine);
       // stage sums beyond 2^60 ns are out of range (a chunk adds less than 2^61, so nothing has wrapped yet)
       if (ser - comp_sum > (2LL << 60) || comp_sum > (1LL << 60)) { bad = 1; break; }
-      long long cmb_mine = 0;
-      for (int q = 0; q < kend; ++q) {
-        const long long leg = __shfl_sync(FULL, leg_mine, q);
-        const long long comp = __shfl_sync(FULL, comp_mine, q);
-        dsp += leg;
-        if (k0 + q == 0) dsp1 = dsp;
-        cmp = max(dsp, cmp) + comp;
-        cmb = max(cmp, cmb) + leg;
-        if (PREFIX && lane == q) cmb_mine = cmb;
-      }
+      // lane q gets the three stage times after matching k0+q; lanes beyond the chunk carry identity maps
+      const long long dsp_mine = dsp + prefix_sum64(leg_mine, lane);
+      MaxPlus f;
+      f.p = comp_mine;
+      f.q = mine ? dsp_mine + comp_mine : MAXPLUS_NONE;
+      f = maxplus_scan(f, lane);
+      const long long cmp_mine = max(cmp + f.p, f.q);
+      MaxPlus h;
+      h.p = leg_mine;
+      h.q = mine ? cmp_mine + leg_mine : MAXPLUS_NONE;
+      h = maxplus_scan(h, lane);
+      const long long cmb_mine = max(cmb + h.p, h.q);
+      if (k0 == 0) dsp1 = __shfl_sync(FULL, dsp_mine, 0);
+      dsp = __shfl_sync(FULL, dsp_mine, kend - 1);
+      cmp = __shfl_sync(FULL, cmp_mine, kend - 1);
+      cmb = __shfl_sync(FULL, cmb_mine, kend - 1);
       if constexpr (PREFIX) {
-        long long run = served_mine;   // inclusive prefix sum over the lanes
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const long long up = __shfl_up_sync(FULL, run, o);
-          if (lane >= o) run += up;
-        }
+        const long long run = prefix_sum64(served_mine, lane);   // inclusive prefix sum over the lanes
         if (mine) {
           prefix_overlap[(size_t)b * k_stride + k0 + lane] = JOBS ? leg_mine : cmb_mine;
           prefix_unserved[(size_t)b * k_stride + k0 + lane] = JOBS ? comp_mine : total - (served_sum + run);
