@@ -163,6 +163,7 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       freerows[w] = N >= lo + 32 ? 0xffffffffu : (N <= lo ? 0u : (0xffffffffu >> (lo + 32 - N)));
     }
 
+    unsigned pace_seen = 0u;   // the largest figure seen at the last look
     while (nnz > 0 && k < k_max) {
       if constexpr (PACE) {
         if ((k & (PACE_EVERY - 1)) == 0) {
@@ -179,8 +180,11 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
             if ((unsigned)(v >> 32) == pace_launch) left = (unsigned)v;
           }
           left = __reduce_max_sync(FULL, left);   // the most entries left among the warps of this scheduler
-          if (left > (unsigned)nnz + PACE_SLACK)
+          // (a figure that has not moved since the last look is not slept on twice: an entry orphaned by a warp
+          // whose slot changed under preemption must not hold the others back)
+          if (left > (unsigned)nnz + PACE_SLACK && left != pace_seen)
             __nanosleep(min((left - (unsigned)nnz - PACE_SLACK) * PACE_NS_PER_ENTRY, PACE_NS_MAX));
+          pace_seen = left;
         }
       }
       // re-match the free rows: a single row that lost its entry is re-matched canonically at once
