@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(128) eval_kernel(int B, int N, int S, const in
               if (lane == q) served_mine = sv_all;
             }
           }
-          __syncwarp();
+          // (no barrier here: a lane only ever touches the rows it owns; the sums after the loop have their own)
         }
       }
       if (bad) break;
