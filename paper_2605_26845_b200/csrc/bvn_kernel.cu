@@ -262,7 +262,8 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
       for (int w = 0; w < W; ++w) freerows[w] = __reduce_or_sync(FULL, gone[w]);
       // unmatch the rows whose entry vanished
       M.release(freerows);
-      __syncwarp();
+      // (x[r] was last read, for the permutation row above, by the lane that clears it here; the barrier after the
+      // loop makes the cleared entries visible to the other lanes, whose later updates of x are made by every lane)
 #pragma unroll
       for (int q = 0; q < W; ++q) {   // lane l looks after rows l, l + 32, ...
         const int r = q * 32 + lane;

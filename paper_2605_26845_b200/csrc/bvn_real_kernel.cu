@@ -176,7 +176,8 @@ __global__ void __launch_bounds__(128) bvn_real_kernel(int B, int N, int S, cons
 #pragma unroll
       for (int w = 0; w < W; ++w) freerows[w] = __reduce_or_sync(FULL, gone[w]);
       M.release(freerows);
-      __syncwarp();
+      // (x[r] was last read, for the permutation row above, by the lane that clears it here; the barrier after the
+      // loop makes the cleared entries visible to the other lanes, whose later updates of x are made by every lane)
 #pragma unroll
       for (int q = 0; q < W; ++q) {
         const int r = q * 32 + lane;

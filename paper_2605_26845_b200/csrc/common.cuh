@@ -835,14 +835,22 @@ __device__ __forceinline__ void record_search(int lane, int i, const unsigned (&
   if constexpr (!CanonMemo<W>::IN_REGS) __syncwarp();
 }
 
-// One row set of the search history (W words at hist + level * W): written by one lane, with a
-// single 8-byte store when the set has two words.
+// One row set of the search history (W words at hist + level * W). The set is uniform and EVERY lane stores
+// it (same address, same value: one shared-memory transaction), so that a lane which reads the history later
+// reads what it wrote itself, in program order: no warp barrier is needed between the store and the loads. The
+// matching x[] is kept the same way (every lane makes every update). Two words go in one 8-byte store, four
+// or eight in 16-byte stores (hist is 16-byte aligned and W * 4 divides 16 or is a multiple of it).
 template <int W>
-__device__ __forceinline__ void hist_store(unsigned* hist, int level, const unsigned (&F)[W], int lane) {
+__device__ __forceinline__ void hist_store(unsigned* hist, int level, const unsigned (&F)[W], int /*lane*/) {
   if constexpr (W == 2) {
-    if (lane == 0) *reinterpret_cast<uint2*>(hist + level * 2) = make_uint2(F[0], F[1]);
+    *reinterpret_cast<uint2*>(hist + level * 2) = make_uint2(F[0], F[1]);
+  } else if constexpr (W % 4 == 0) {
+#pragma unroll
+    for (int q = 0; q < W; q += 4)
+      *reinterpret_cast<uint4*>(hist + level * W + q) = make_uint4(F[q], F[q + 1], F[q + 2], F[q + 3]);
   } else {
-    if (lane < W) hist[level * W + lane] = pick<W>(F, lane);
+#pragma unroll
+    for (int w = 0; w < W; ++w) hist[level * W + w] = F[w];
   }
 }
 template <int W>
@@ -944,7 +952,6 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
       for (int w = 0; w < W; ++w) work[WK_POP] += __popc(F[w]);
       hist_store<W>(hist, level, F, lane);
     }
-    __syncwarp();
     // lowest column row i may take (its own column always qualifies)
     int jstar, cur, L, sl;   // the column, the row that gives it up, its lane and slot
     if (!lowest_qualifying_column<CPL>(
@@ -975,15 +982,14 @@ __device__ __forceinline__ bool canonicalise(int N, int lane, int start, int las
           break;
         }
         if (lane == L2) M.assign(s2, cur);
-        if (lane == 0) x[MS_AT(cur, N)] = (short)c2;
+        x[MS_AT(cur, N)] = (short)c2;   // every lane (see hist_store)
         last = max(last, cur);
         cur = nxt;
         --lvl;
         work[WK_ROT]++;
       }
       if (lane == L) M.assign(sl, i);
-      if (lane == 0) x[MS_AT(i, N)] = (short)jstar;
-      __syncwarp();
+      x[MS_AT(i, N)] = (short)jstar;
       if constexpr (MEMO) {
         // the moved rows changed column: every record that contains one of them is void
         unsigned hit[W];
@@ -1084,10 +1090,8 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
     const int L = j / CPL, sl = j % CPL;
     const int i = __shfl_sync(FULL, pick<CPL>(par, sl), L);
     const int jprev = x[MS_AT(i, N)];
-    __syncwarp();
     if (lane == L) M.assign(sl, i);
-    if (lane == 0) x[MS_AT(i, N)] = (short)j;
-    __syncwarp();
+    x[MS_AT(i, N)] = (short)j;   // every lane (see hist_store)
     lo = min(lo, i);
     hi = max(hi, i);
     set_bit<W>(changed, i);
@@ -1157,14 +1161,13 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
       if (M.mr[s] >= 0 && M.in(nw, s)) front |= 1u << s;
     freeable |= front;
   }
-  __syncwarp();
   // the lowest column that r0 is adjacent to and that can be released
   int c0, cur, L, sl;   // the column, the row that gives it up, its lane and slot
   if (!lowest_qualifying_column<CPL>(
           lane, M, [&](int s) { return ((freeable >> s) & 1u) && intersects<W>(C[s], r0mask); }, c0, cur, L, sl))
     return 0;
   if (lane == L) M.assign(sl, r0);
-  if (lane == 0) x[MS_AT(r0, N)] = (short)c0;
+  x[MS_AT(r0, N)] = (short)c0;   // every lane (see hist_store)
   set_bit<W>(changed, r0);
   hi = max(hi, r0);
   if (cur < 0) return 1;   // r0 took the free column itself
@@ -1188,11 +1191,11 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
     }
     if (!found) return -1;
     if (lane == L2) M.assign(s2, cur);
-    if (lane == 0) x[MS_AT(cur, N)] = (short)c2;
+    x[MS_AT(cur, N)] = (short)c2;
     set_bit<W>(changed, cur);
     hi = max(hi, cur);
     work[WK_AUG]++;
-    if (lvl == 1) { __syncwarp(); return 1; }
+    if (lvl == 1) return 1;
     if (nxt < 0) return -1;
     cur = nxt;
     --lvl;

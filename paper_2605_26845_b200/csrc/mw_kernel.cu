@@ -97,7 +97,7 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
     const int owner = __shfl_sync(FULL, st.M.row_of(sl), L);
     if (owner < 0) {
       if (lane == L) st.M.assign(sl, r);
-      if (lane == 0) x[r] = (short)(L * CPL + sl);
+      x[r] = (short)(L * CPL + sl);   // every lane: a lane later reads what it wrote itself (see hist_store)
     } else {
       set_bit<W>(freerows, r);
     }
@@ -181,10 +181,8 @@ __device__ __forceinline__ bool solve_assignment(const View& R, int N, int lane,
       const int L = j / CPL, sl = j % CPL;
       const int i = __shfl_sync(FULL, pick<CPL>(pred, sl), L);
       const int jprev = x[MS_AT(i, N)];
-      __syncwarp();
       if (lane == L) st.M.assign(sl, i);
-      if (lane == 0) x[MS_AT(i, N)] = (short)j;
-      __syncwarp();
+      x[MS_AT(i, N)] = (short)j;   // every lane
       if (i == f) break;
       j = jprev;
       if (j < 0) { ok = false; break; }
