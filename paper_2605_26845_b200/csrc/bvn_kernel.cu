@@ -194,11 +194,16 @@ __global__ void __launch_bounds__(128) bvn_kernel(int B, int N, int S, const int
         for (int it = 0; it < N; ++it) {
           const int r0 = lowest_bit<W>(freerows);
           if (r0 < 0) break;
-          const int rc = canonical_repair<CPL>(N, lane, r0, C, M, x, hist, hi_changed, memo.changed, work);
+          int single = 0;
+#pragma unroll
+          for (int w = 0; w < W; ++w) single += __popc(freerows[w]);
+          const int rc = canonical_repair<CPL>(N, lane, r0, C, M, x, hist, hi_changed, memo.changed, work, single == 1,
+                                               lo_changed);
           if (rc < 0) { okm = false; break; }
           if (rc == 0) { work[WK_BATCH]++; break; }   // needs rows below r0: the general search below takes over
-          work[WK_TIGHT]++;
           clear_bit<W>(freerows, r0);
+          if (rc == 2) { work[WK_BATCH]++; break; }   // rows below r0 had to move: the window starts at the lowest of them
+          work[WK_TIGHT]++;
           lo_changed = min(lo_changed, r0 + 1);   // row r0 has its final column; the rows that moved lie above it
         }
         if (!okm) { st_code = MOESCHED_ST_INTERNAL; break; }

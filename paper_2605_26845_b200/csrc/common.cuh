@@ -1115,12 +1115,17 @@ __device__ __forceinline__ bool augment_from(int N, int lane, int f, const unsig
 // matchings that leave the other free rows out, hence also among the complete ones if the rest can still be
 // matched above it; if not, the caller's general search lowers the window as far as it has to.) This replaces an arbitrary augmenting path followed by a search (and
 // usually a rotation) for row r0. Returns 1 when done (hi = highest row moved, `changed` gets the moved rows),
-// 0 when r0 cannot be re-matched without rows below it (the caller falls back to augment_from), -1 if an
-// iteration limit was hit.
+// 0 when r0 cannot be re-matched this way (the caller falls back to augment_from), -1 if an iteration limit
+// was hit.
+// With `may_lower` (the caller passes it when r0 is the only free row) the search does not give up when r0 is
+// adjacent to no column that the rows above it can release: it admits the highest row BELOW r0 that is adjacent
+// to a releasable column, continues from that row's column, and repeats until r0 can be served. The path then
+// disturbs as few low rows as possible (as augment_from's does); r0's column is no longer final, `lo` is lowered
+// to the lowest row that moved, and 2 is returned.
 template <int CPL>
 __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const unsigned (&C)[CPL][CPL], Match<CPL>& M,
                                                 short* x, unsigned* hist, int& hi, unsigned (&changed)[CPL],
-                                                unsigned (&work)[MOESCHED_WORK_FIELDS]) {
+                                                unsigned (&work)[MOESCHED_WORK_FIELDS], bool may_lower, int& lo) {
   constexpr int W = CPL;
   unsigned alive[W], r0mask[W];
   ge_mask<W>(r0 + 1, alive);        // rows above r0 not reached yet
@@ -1132,6 +1137,16 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
   if (__ballot_sync(FULL, front != 0u) == 0u) return 0;   // no free column: nothing to hand out
   unsigned freeable = front;        // bit s: column s is free or can be released
   int level = 0;
+  bool lowered = false;
+  unsigned below[W];                // rows below r0 not admitted yet
+  {
+    unsigned from_r0[W];
+    ge_mask<W>(r0, from_r0);
+#pragma unroll
+    for (int w = 0; w < W; ++w) below[w] = ~from_r0[w];
+  }
+  int c0 = -1, cur = -1, L = 0, sl = 0;   // r0's column, the row that gives it up, its lane and slot
+  for (int round = 0; round <= N; ++round) {
   for (int it = 0; it < N; ++it) {
     unsigned acc[W];
 #pragma unroll
@@ -1162,10 +1177,41 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
     freeable |= front;
   }
   // the lowest column that r0 is adjacent to and that can be released
-  int c0, cur, L, sl;   // the column, the row that gives it up, its lane and slot
-  if (!lowest_qualifying_column<CPL>(
+  if (lowest_qualifying_column<CPL>(
           lane, M, [&](int s) { return ((freeable >> s) & 1u) && intersects<W>(C[s], r0mask); }, c0, cur, L, sl))
-    return 0;
+    break;
+  c0 = -1;
+  if (!may_lower) return 0;
+  // admit the highest row below r0 that could move to a releasable column
+  unsigned acc[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+  for (int s = 0; s < CPL; ++s) {
+    if ((freeable >> s) & 1u) {
+#pragma unroll
+      for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
+    }
+  }
+  unsigned waiting[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) waiting[w] = __reduce_or_sync(FULL, acc[w]) & below[w];
+  const int t = highest_bit<W>(waiting);
+  if (t < 0) return 0;
+  clear_bit<W>(below, t);
+  lowered = true;
+  unsigned tmask[W];
+  onehot_mask<W>(t, tmask);
+  ++level;
+  hist_store<W>(hist, level, tmask, lane);
+  front = 0u;
+#pragma unroll
+  for (int s = 0; s < CPL; ++s)
+    if (M.mr[s] >= 0 && M.in(tmask, s)) front |= 1u << s;
+  freeable |= front;
+  work[WK_SCAN]++;
+  }
+  if (c0 < 0) return -1;
   if (lane == L) M.assign(sl, r0);
   x[MS_AT(r0, N)] = (short)c0;   // every lane (see hist_store)
   set_bit<W>(changed, r0);
@@ -1173,6 +1219,42 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
   if (cur < 0) return 1;   // r0 took the free column itself
   int lvl = level_of_row<W>(hist, level, MS_AT(cur, N), lane);
   if (lvl == 0) return -1;
+  if (lowered) {
+    // An admitted row joined through a column of ANY earlier level, so a row moves to the lowest column it is
+    // adjacent to whose row was reached at an earlier level (or that is free); the levels still fall strictly.
+    lo = min(lo, r0);
+    for (int it = 0; it <= N; ++it) {
+      unsigned cmask[W], Hm[W];
+      onehot_mask<W>(cur, cmask);
+#pragma unroll
+      for (int w = 0; w < W; ++w) Hm[w] = 0u;
+      for (int d = 1; d < lvl; ++d) {
+        unsigned Hd[W];
+        hist_load<W>(hist, d, Hd);
+#pragma unroll
+        for (int w = 0; w < W; ++w) Hm[w] |= Hd[w];
+      }
+      int c2, nxt, L2, s2;
+      if (!lowest_qualifying_column<CPL>(
+              lane, M,
+              [&](int s) {
+                return lane * CPL + s < N && (M.mr[s] < 0 || M.in(Hm, s)) && intersects<W>(C[s], cmask);
+              },
+              c2, nxt, L2, s2))
+        return -1;
+      if (lane == L2) M.assign(s2, cur);
+      x[MS_AT(cur, N)] = (short)c2;
+      set_bit<W>(changed, cur);
+      hi = max(hi, cur);
+      lo = min(lo, cur);
+      work[WK_AUG]++;
+      if (nxt < 0) return 2;   // took the free column
+      cur = nxt;
+      lvl = level_of_row<W>(hist, level, MS_AT(cur, N), lane);
+      if (lvl == 0) return -1;
+    }
+    return -1;
+  }
   for (int it = 0; it <= N; ++it) {
     // cur, reached at level lvl, moves to a column of level lvl - 1 (level 0: the free column)
     unsigned cmask[W];
