@@ -156,8 +156,13 @@ int moesched_mw_decompose(int B, int N, const int32_t* d_demand, int k_max, uint
  *                   canonically at once, 3 canonicalisation sweeps that searched,
  *                   4 search levels, 5 rotation steps, 6 matchings, 7 rows
  *                   skipped as unchanged prefix, 8 rows expanded by the
- *                   canonicalisation searches (frontier pops), 9 canonical
- *                   re-matchings that had to fall back to the general search
+ *                   canonicalisation searches (frontier pops), 9 re-matchings
+ *                   that needed rows below the row whose entry vanished
+ * A batch that is resident on the GPU all at once (from 12 matrices per SM up, with
+ * scratch, without d_work) is launched with its warps pacing one another through a
+ * 128 KB table built into the library (a warp that is ahead sleeps for a moment). This
+ * changes timing only, never results; entries carry the launch's number, so calls that
+ * overlap on one GPU merely ignore each other's entries.
  */
 int moesched_bvn_decompose(int B, int N, const int32_t* d_demand, int k_max, uint8_t* d_perm,
                            int32_t* d_coef, int32_t* d_count, int32_t* d_aug, int32_t* d_scratch,
