@@ -1167,7 +1167,24 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
     for (int w = 0; w < W; ++w) below[w] = ~from_r0[w];
   }
   int c0 = -1, cur = -1, L = 0, sl = 0;   // r0's column, the row that gives it up, its lane and slot
-  for (int round = 0; round <= N; ++round) {
+  // The lowest column r0 is adjacent to that is free or whose row lies above r0: if that row is reached, r0 can
+  // have nothing lower and the search stops there (with one or two columns per lane, where finding it pays).
+  constexpr bool EARLY = CPL <= 2;
+  unsigned target[W];
+#pragma unroll
+  for (int w = 0; w < W; ++w) target[w] = 0u;
+  int early = 0;
+  int tc = -1, trow = -1, tL = 0, tsl = 0;   // that column, its row, lane and slot
+  if constexpr (EARLY) {
+    if (lowest_qualifying_column<CPL>(
+            lane, M,
+            [&](int s) { return lane * CPL + s < N && (M.mr[s] < 0 || M.mr[s] > r0) && intersects<W>(C[s], r0mask); },
+            tc, trow, tL, tsl)) {
+      if (trow >= 0) onehot_mask<W>(trow, target);
+      else early = -1;   // the free column itself: nothing to search
+    }
+  }
+  for (int round = 0; round <= N && early == 0; ++round) {
   for (int it = 0; it < N; ++it) {
     unsigned acc[W];
 #pragma unroll
@@ -1190,6 +1207,9 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
     work[WK_SCAN]++;
     if (!grew) break;
     ++level;
+    if constexpr (EARLY) {
+      if (intersects<W>(nw, target)) { early = level; break; }
+    }
     hist_store<W>(hist, level, nw, lane);
     front = 0u;
 #pragma unroll
@@ -1197,7 +1217,8 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
       if (M.mr[s] >= 0 && M.in(nw, s)) front |= 1u << s;
     freeable |= front;
   }
-  // the lowest column that r0 is adjacent to and that can be released
+  if (early != 0) break;
+  // otherwise the lowest column that r0 is adjacent to and that can be released
   if (lowest_qualifying_column<CPL>(
           lane, M, [&](int s) { return ((freeable >> s) & 1u) && intersects<W>(C[s], r0mask); }, c0, cur, L, sl))
     break;
@@ -1232,13 +1253,14 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
   freeable |= front;
   work[WK_SCAN]++;
   }
+  if (early != 0) { c0 = tc; cur = trow; L = tL; sl = tsl; }
   if (c0 < 0) return -1;
   if (lane == L) M.assign(sl, r0);
   x[MS_AT(r0, N)] = (short)c0;   // every lane (see hist_store)
   set_bit<W>(changed, r0);
   hi = max(hi, r0);
   if (cur < 0) return 1;   // r0 took the free column itself
-  int lvl = level_of_row<W>(hist, level, MS_AT(cur, N), lane);
+  int lvl = early > 0 ? early : level_of_row<W>(hist, level, MS_AT(cur, N), lane);
   if (lvl == 0) return -1;
   if (lowered) {
     // An admitted row joined through a column of ANY earlier level, so a row moves to the lowest column it is
