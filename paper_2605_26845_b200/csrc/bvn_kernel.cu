@@ -35,7 +35,7 @@ constexpr unsigned PACE_NS_PER_ENTRY = 2000, PACE_NS_MAX = 200000;
 __device__ unsigned long long g_pace[256][64];   // [SM][warp slot] = launch number << 32 | entries left
 
 template <int CPL, int MODE, bool COUNT, bool PACE = false>
-__global__ void __launch_bounds__(128, CPL <= 2 ? 7 : 1) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
+__global__ void __launch_bounds__(128, CPL <= 2 ? 7 : 0) bvn_kernel(int B, int N, int S, const int32_t* __restrict__ demand, int k_max,
                                                   uint8_t* __restrict__ perm, int32_t* __restrict__ coef,
                                                   int32_t* __restrict__ count, int32_t* __restrict__ aug,
                                                   int32_t* scratch, int32_t* __restrict__ status,
