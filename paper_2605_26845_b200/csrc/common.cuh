@@ -1185,73 +1185,73 @@ __device__ __forceinline__ int canonical_repair(int N, int lane, int r0, const u
     }
   }
   for (int round = 0; round <= N && early == 0; ++round) {
-  for (int it = 0; it < N; ++it) {
+    for (int it = 0; it < N; ++it) {
+      unsigned acc[W];
+#pragma unroll
+      for (int w = 0; w < W; ++w) acc[w] = 0u;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s) {
+        if ((front >> s) & 1u) {
+#pragma unroll
+          for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
+        }
+      }
+      unsigned nw[W];
+      bool grew = false;
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        nw[w] = __reduce_or_sync(FULL, acc[w]) & alive[w];
+        alive[w] &= ~nw[w];
+        grew |= nw[w] != 0u;
+      }
+      work[WK_SCAN]++;
+      if (!grew) break;
+      ++level;
+      if constexpr (EARLY) {
+        if (intersects<W>(nw, target)) { early = level; break; }
+      }
+      hist_store<W>(hist, level, nw, lane);
+      front = 0u;
+#pragma unroll
+      for (int s = 0; s < CPL; ++s)
+        if (M.mr[s] >= 0 && M.in(nw, s)) front |= 1u << s;
+      freeable |= front;
+    }
+    if (early != 0) break;
+    // otherwise the lowest column that r0 is adjacent to and that can be released
+    if (lowest_qualifying_column<CPL>(
+            lane, M, [&](int s) { return ((freeable >> s) & 1u) && intersects<W>(C[s], r0mask); }, c0, cur, L, sl))
+      break;
+    c0 = -1;
+    if (!may_lower) return 0;
+    // admit the highest row below r0 that could move to a releasable column
     unsigned acc[W];
 #pragma unroll
     for (int w = 0; w < W; ++w) acc[w] = 0u;
 #pragma unroll
     for (int s = 0; s < CPL; ++s) {
-      if ((front >> s) & 1u) {
+      if ((freeable >> s) & 1u) {
 #pragma unroll
         for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
       }
     }
-    unsigned nw[W];
-    bool grew = false;
+    unsigned waiting[W];
 #pragma unroll
-    for (int w = 0; w < W; ++w) {
-      nw[w] = __reduce_or_sync(FULL, acc[w]) & alive[w];
-      alive[w] &= ~nw[w];
-      grew |= nw[w] != 0u;
-    }
-    work[WK_SCAN]++;
-    if (!grew) break;
+    for (int w = 0; w < W; ++w) waiting[w] = __reduce_or_sync(FULL, acc[w]) & below[w];
+    const int t = highest_bit<W>(waiting);
+    if (t < 0) return 0;
+    clear_bit<W>(below, t);
+    lowered = true;
+    unsigned tmask[W];
+    onehot_mask<W>(t, tmask);
     ++level;
-    if constexpr (EARLY) {
-      if (intersects<W>(nw, target)) { early = level; break; }
-    }
-    hist_store<W>(hist, level, nw, lane);
+    hist_store<W>(hist, level, tmask, lane);
     front = 0u;
 #pragma unroll
     for (int s = 0; s < CPL; ++s)
-      if (M.mr[s] >= 0 && M.in(nw, s)) front |= 1u << s;
+      if (M.mr[s] >= 0 && M.in(tmask, s)) front |= 1u << s;
     freeable |= front;
-  }
-  if (early != 0) break;
-  // otherwise the lowest column that r0 is adjacent to and that can be released
-  if (lowest_qualifying_column<CPL>(
-          lane, M, [&](int s) { return ((freeable >> s) & 1u) && intersects<W>(C[s], r0mask); }, c0, cur, L, sl))
-    break;
-  c0 = -1;
-  if (!may_lower) return 0;
-  // admit the highest row below r0 that could move to a releasable column
-  unsigned acc[W];
-#pragma unroll
-  for (int w = 0; w < W; ++w) acc[w] = 0u;
-#pragma unroll
-  for (int s = 0; s < CPL; ++s) {
-    if ((freeable >> s) & 1u) {
-#pragma unroll
-      for (int w = 0; w < W; ++w) acc[w] |= C[s][w];
-    }
-  }
-  unsigned waiting[W];
-#pragma unroll
-  for (int w = 0; w < W; ++w) waiting[w] = __reduce_or_sync(FULL, acc[w]) & below[w];
-  const int t = highest_bit<W>(waiting);
-  if (t < 0) return 0;
-  clear_bit<W>(below, t);
-  lowered = true;
-  unsigned tmask[W];
-  onehot_mask<W>(t, tmask);
-  ++level;
-  hist_store<W>(hist, level, tmask, lane);
-  front = 0u;
-#pragma unroll
-  for (int s = 0; s < CPL; ++s)
-    if (M.mr[s] >= 0 && M.in(tmask, s)) front |= 1u << s;
-  freeable |= front;
-  work[WK_SCAN]++;
+    work[WK_SCAN]++;
   }
   if (early != 0) { c0 = tc; cur = trow; L = tL; sl = tsl; }
   if (c0 < 0) return -1;
